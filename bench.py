@@ -222,20 +222,26 @@ def run_ours(args):
     assert ctx.kv_sync_status(stream) == 0
     computed, n_chunks, launches_per_step = plan["computed"], plan["chunks"], plan["launches"]
 
-    # ---- timed region: device time of K steps, per-kernel events on ----
-    assert ctx.kv_set_option("profile", 1) == 0
+    # ---- timed region: device time of K steps (per-kernel events off) ----
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    kinds = {k: [0.0, 0] for k in kb.KINDS}
     e0.record(stream)
     for _ in range(args.steps):
-        step(kinds)
+        step()
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
     dev_ms = e0.elapsed_time(e1)
+    assert ctx.kv_sync_status(stream) == 0
+
+    # ---- per-kernel breakdown: separate steps with an event pair around every launch ----
+    prof_steps = max(1, min(args.steps, args.profile_steps))
+    assert ctx.kv_set_option("profile", 1) == 0
+    kinds = {k: [0.0, 0] for k in kb.KINDS}
+    for _ in range(prof_steps):
+        step(kinds)
     assert ctx.kv_sync_status(stream) == 0
     assert ctx.kv_set_option("profile", 0) == 0
 
@@ -292,15 +298,15 @@ def run_ours(args):
         total_flops = sum(fl.values())
         step_s = dev_s / args.steps
         gemm_kinds = ("qkv_gemm", "o_gemm", "gateup_gemm", "down_gemm")
-        gemm_ms = sum(kinds[k][0] for k in gemm_kinds) / args.steps
-        gemm_launches = sum(kinds[k][1] for k in gemm_kinds) // args.steps
+        gemm_ms = sum(kinds[k][0] for k in gemm_kinds) / prof_steps
+        gemm_launches = sum(kinds[k][1] for k in gemm_kinds) // prof_steps
         gemm_tf = sum(fl[k] for k in gemm_kinds) / (gemm_ms * 1e-3) / 1e12 if gemm_ms else None
         peak = peaks["bf16_tflops_sustained"]
         breakdown = {}
         for k, (ms, n) in kinds.items():
-            ent = {"ms_per_step": ms / args.steps, "launches_per_step": n // args.steps}
+            ent = {"ms_per_step": ms / prof_steps, "launches_per_step": n // prof_steps}
             if k in fl and ms:
-                ent["tflops"] = fl[k] / (ms / args.steps * 1e-3) / 1e12
+                ent["tflops"] = fl[k] / (ms / prof_steps * 1e-3) / 1e12
             breakdown[k] = ent
         traffic = None
         tp = os.path.join(ROOT, "profiles", "traffic.json")
@@ -335,6 +341,10 @@ def run_ours(args):
                          "frac": gemm_tf / peak if gemm_tf else None, "peak_kind": f"sustained, {peaks['source']}",
                          "launches_per_step": gemm_launches, "traffic": traffic},
             "kernels": breakdown,
+            "timing": {"value_steps": args.steps, "value_profile_option": 0,
+                       "kernels_steps": prof_steps, "kernels_profile_option": 1,
+                       "note": "value/ms_per_step: one event pair around all steps; kernels/roofline: separate steps "
+                               "with an event pair around every launch"},
             "aux": {"arena_flush": {"bytes": int(arena.numel() * 2), "gbs": flush_gbs, "peak_gbs": peaks["hbm_gbs"],
                                     "frac": flush_gbs / peaks["hbm_gbs"], "note": "write-only fill; peak is a read+write copy"},
                     "health_probe_status": int(st_probe),
@@ -408,6 +418,8 @@ def main():
     ap.add_argument("--config", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--chunk", type=int, default=None,
                     help="tokens per workspace chunk (default: synth.BENCH_CHUNK_TOKENS = 18944)")
+    ap.add_argument("--profile-steps", type=int, default=2,
+                    help="steps of the separate per-kernel timing pass (at most --steps)")
     ap.add_argument("--cpu-tokens", type=int, default=256)
     ap.add_argument("--ref-tokens", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")

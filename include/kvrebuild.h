@@ -141,8 +141,8 @@ int kv_rebuild(kvr_ctx *ctx, const kv_weights *weights, const int32_t *token_pre
                const int32_t *prefix_lens, const int32_t *block_tables, int32_t n_requests,
                int32_t max_blocks_per_req, void *stream);
 
-/* The paper's stated future work (Sec. 4.2: recovering the pool "without refilling would
- * require fine-grained consistency tracking"): a caller that has verified the first
+/* Paper Sec. 4.2 (future work: reuse of pool contents instead of a full refill, which needs the
+ * caller to track which rows are still consistent): a caller that has verified the first
  * valid_lens[r] rows of request r in the arena (for example a shared prompt whose other
  * sharers are alive) rebuilds only the tail.  Same as kv_rebuild except that tokens
  * [0, valid_lens[r]) are neither recomputed nor written -- their rows stay byte-identical --
@@ -184,7 +184,12 @@ int kv_readback_dev(kvr_ctx *ctx, int32_t layer, const int32_t *block_table_host
  *   - The staging array (16 KiB + 2 x 2 MiB) is held by every GPU that loads
  *     the library until the process exits.
  *   - The first call on a device looks up the array's device address
- *     (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *     (cudaGetSymbolAddress).  Every call copies from pageable host memory and
+ *     waits for the stream before it returns, so no call, first or later, may be
+ *     issued while `stream` is being captured.
+ *   - The layer's K and V planes must lie inside the device allocation that
+ *     holds arena_dev (its extent is queried from the driver); a geometry that
+ *     reaches past it returns KVR_ERR_INVALID_ARG and reads nothing.
  *   - All calls share the one array and it keeps the previous call's bytes;
  *     nothing in it has to start at zero because every byte read back is
  *     written first.  Two calls that overlap in time on one GPU (different
@@ -211,16 +216,18 @@ int kv_readback_noalloc(const void *arena_dev, const kv_arena_geometry *geom, in
 int kv_resume_logits(kvr_ctx *ctx, const void *final_gain_dev, const void *lm_head_dev, float *logits_out_dev,
                      void *stream);
 
-/* Paper Sec. 4.2 step 2 ("flushes the KV-cache pool"; the pool is invalidated and starts a new
- * epoch): overwrite every byte of the bound arena with the 32-bit word `fill_word` (0 for
+/* Paper Sec. 4.2, handover step 2 (pool flush: the old contents are invalidated before any
+ * request is rebuilt): overwrite every byte of the bound arena with the 32-bit word `fill_word` (0 for
  * zeros; any NaN pattern to make stale reads visible).  Enqueues on `stream`; HBM-bound. */
 int kv_arena_flush(kvr_ctx *ctx, uint32_t fill_word, void *stream);
 
-/* Paper Sec. 4.2 step 2 ("checks GPU health with a lightweight CUDA operation"): one small
+/* Paper Sec. 4.2, handover step 2 (GPU health check by a small device operation): one small
  * kernel per call, one 64-thread block per SM; every block runs a fixed xorshift32-plus-increment
  * chain (ALU), sums it through shared memory, publishes the result and a flag to global memory
  * and waits -- for at most timeout_ms, never longer -- until it sees its neighbour block's
- * flag (cross-SM visibility).  The host waits for the kernel for at most 2 x timeout_ms.
+ * flag (cross-SM visibility).  The flag word is a per-context call counter, so flags left by an
+ * earlier call (same seed or not) never satisfy a later call's wait.  The host waits for the
+ * kernel for at most 2 x timeout_ms.
  *   KVR_OK                   every block finished, every wait was met, *checksum_out (if not
  *                            NULL) = XOR over blocks b of rotl(result_b, b % 32)
  *   KVR_ERR_DEVICE_TIMEOUT   a device wait ran out or the kernel did not finish in time

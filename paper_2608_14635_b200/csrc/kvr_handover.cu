@@ -32,8 +32,11 @@ __device__ __forceinline__ uint32_t xorshift32(uint32_t x) {
     return x;
 }
 
-__global__ void __launch_bounds__(PROBE_THREADS) probe_kernel(uint32_t seed, uint32_t *flags, uint32_t *out,
-                                                              int *status, long long limit_cycles, int publish) {
+// `epoch` is a word no earlier probe of this flag array has published (the context counts its
+// calls), so a flag left behind by a previous call can never satisfy this call's wait.
+__global__ void __launch_bounds__(PROBE_THREADS) probe_kernel(uint32_t seed, uint32_t epoch, uint32_t *flags,
+                                                              uint32_t *out, int *status, long long limit_cycles,
+                                                              int publish) {
     __shared__ uint32_t red[PROBE_THREADS];
     const uint32_t b = blockIdx.x, t = threadIdx.x;
     uint32_t x = seed ^ (b * 0x9E3779B9u) ^ (t * 0x85EBCA6Bu);
@@ -48,12 +51,12 @@ __global__ void __launch_bounds__(PROBE_THREADS) probe_kernel(uint32_t seed, uin
     if (t == 0) {
         out[b] = red[0];
         __threadfence();
-        if (publish) atomicExch(&flags[b], seed | 1u);
+        if (publish) atomicExch(&flags[b], epoch);
         // the neighbour block must become visible within the limit; a wait that runs out
         // is reported through the status word, never by spinning on
         const uint32_t nb = (b + 1) % gridDim.x;
         const long long t0 = clock64();
-        while (atomicAdd(&flags[nb], 0u) != (seed | 1u)) {
+        while (atomicAdd(&flags[nb], 0u) != epoch) {
             if (clock64() - t0 > limit_cycles) {
                 atomicExch(status, KVR_ERR_DEVICE_TIMEOUT);
                 break;
@@ -74,9 +77,9 @@ int launch_arena_flush(void *arena, size_t bytes, uint32_t word, int n_sms, cuda
     return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
 }
 
-int launch_probe(uint32_t seed, uint32_t *flags, uint32_t *out, int *status, int blocks, long long limit_cycles,
-                 int publish, cudaStream_t s) {
-    probe_kernel<<<blocks, PROBE_THREADS, 0, s>>>(seed, flags, out, status, limit_cycles, publish);
+int launch_probe(uint32_t seed, uint32_t epoch, uint32_t *flags, uint32_t *out, int *status, int blocks,
+                 long long limit_cycles, int publish, cudaStream_t s) {
+    probe_kernel<<<blocks, PROBE_THREADS, 0, s>>>(seed, epoch, flags, out, status, limit_cycles, publish);
     return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
 }
 

@@ -65,6 +65,7 @@ struct kvr_ctx {
     // options
     int gemm_impl = 2, attn_impl = 2, profile = 0, probe_mute = 0;
     uint32_t *d_probe = nullptr;   // [2 * PROBE_MAX_BLOCKS]: flags, results
+    uint32_t probe_epoch = 0;      // word the current probe publishes; never 0, never reused by the next call
     int clock_khz = 0;
     // per-launch event pairs of the last call (profile mode)
     std::vector<cudaEvent_t> ev_pool;
@@ -551,6 +552,10 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     if (R > c->max_req || width > c->max_blk) return KVR_ERR_WORKSPACE;
     const bool fp32 = is_fp32(c);
     const bool use_tc_gemm = !fp32 && c->gemm_impl >= 1;
+    // The fused QKV epilogue hands every 128-column half tile to exactly one of q, k, v, so it needs
+    // q_dim and kv_dim to be multiples of 128; other head counts take the plain projection + RoPE/scatter
+    // kernels for this one step (same arena rows, no tile ever straddles two destinations).
+    const bool use_tc_qkv = use_tc_gemm && md.q_dim % 128 == 0 && md.kv_dim % 128 == 0;
     // tcgen05 attention needs 16-slot blocks (the CTA-pair kernel also head dim 128): the next kernel down takes over
     const bool use_fa2_attn = !fp32 && c->attn_impl == 3 && c->tm_kv_ok && md.hd == 128;
     const bool use_fa_attn = !fp32 && c->attn_impl >= 2 && c->tm_kv_ok;   // either tcgen05 kernel
@@ -691,7 +696,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
             }
             // QKV projection + RoPE + paged store (last layer: K/V only)
             const QkvExtras ex = qkv_extras(c, l);
-            if (use_tc_gemm) {
+            if (use_tc_qkv) {
                 TcGemmEpilogue ep{};
                 set_tc_extras(ep, ex, !last);
                 ep.mode = TC_QKV; ep.M = n; ep.K = md.d;
@@ -872,6 +877,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     const ModelDims &md = c->md;
     const bool fp32 = is_fp32(c);
     const bool use_tc = !fp32 && c->gemm_impl >= 1;
+    const bool use_tc_q = use_tc && md.q_dim % 128 == 0;   // as in the rebuild: whole 128-column halves only
     const bool use_fa = !fp32 && c->attn_impl >= 2 && c->tm_kv_ok;   // one-row tiles: the single-CTA kernel
     const bool use_mma = !fp32 && !use_fa && c->attn_impl != 0;
     if ((use_tc || use_fa || use_mma) && !c->tc_ready) return KVR_ERR_UNSUPPORTED;
@@ -915,7 +921,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     // q of the final tokens (RoPE at position len - 1); their K/V are already in the arena
     QkvExtras ex = qkv_extras(c, l);
     ex.bk = ex.bv = ex.kn = nullptr;   // only q is projected here
-    if (use_tc) {
+    if (use_tc_q) {
         TcGemmEpilogue ep{};
         set_tc_extras(ep, ex, true);
         ep.mode = TC_QKV; ep.M = R; ep.K = md.d; ep.N = md.q_dim;
@@ -1008,7 +1014,8 @@ int kv_health_probe(kvr_ctx *c, uint32_t seed, int32_t timeout_ms, uint32_t *che
     uint32_t *flags = c->d_probe, *out = c->d_probe + PROBE_MAX_BLOCKS;
     cudaEvent_t done;
     CU_OK(cudaEventCreateWithFlags(&done, cudaEventDisableTiming));
-    int st = launch_probe(seed, flags, out, c->d_status, blocks, limit, c->probe_mute ? 0 : 1, s);
+    if (++c->probe_epoch == 0) c->probe_epoch = 1;   // flags start at 0 and hold earlier epochs only
+    int st = launch_probe(seed, c->probe_epoch, flags, out, c->d_status, blocks, limit, c->probe_mute ? 0 : 1, s);
     if (st == KVR_OK && cudaEventRecord(done, s) != cudaSuccess) st = KVR_ERR_CUDA;
     if (st == KVR_OK) {
         // host-side bound: the device waits give up after timeout_ms, so 2 x that is generous

@@ -135,7 +135,7 @@ int launch_attn_fa(const CUtensorMap &tmQ, const CUtensorMap &tmKV, const AttnTi
 // ---- handover device steps (kvr_handover.cu) ----
 constexpr int PROBE_THREADS = 64, PROBE_ITERS = 1000, PROBE_MAX_BLOCKS = 1024;
 int launch_arena_flush(void *arena, size_t bytes, uint32_t word, int n_sms, cudaStream_t s);
-int launch_probe(uint32_t seed, uint32_t *flags, uint32_t *out, int *status, int blocks, long long limit_cycles,
-                 int publish, cudaStream_t s);
+int launch_probe(uint32_t seed, uint32_t epoch, uint32_t *flags, uint32_t *out, int *status, int blocks,
+                 long long limit_cycles, int publish, cudaStream_t s);
 
 }  // namespace kvr

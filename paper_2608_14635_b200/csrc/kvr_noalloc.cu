@@ -73,6 +73,30 @@ extern "C" int kv_readback_noalloc(const void *arena_dev, const kv_arena_geometr
     if (dev < 0 || dev >= MAX_DEVICES) return KVR_ERR_UNSUPPORTED;
     DeviceGuard guard(dev);
     if (!guard.ok) return KVR_ERR_CUDA;
+    {
+        // There is no arena_bytes argument, so the extent of the allocation that holds arena_dev is
+        // asked of the driver (a query, not an allocation): the layer's K and V planes must lie
+        // inside it, otherwise a wrong geometry would turn into an out-of-range device read.
+        typedef CUresult (*RangeFn)(CUdeviceptr *, size_t *, CUdeviceptr);
+        static RangeFn range_fn = nullptr;
+        {
+            std::lock_guard<std::mutex> lock(g_mu);
+            if (!range_fn) {
+                void *fn = nullptr;
+                cudaDriverEntryPointQueryResult qres;
+                if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+                    qres != cudaDriverEntryPointSuccess || !fn)
+                    return KVR_ERR_CUDA;
+                range_fn = (RangeFn)fn;
+            }
+        }
+        CUdeviceptr abase = 0;
+        size_t asize = 0;
+        if (range_fn(&abase, &asize, (CUdeviceptr)(uintptr_t)arena_dev) != CUDA_SUCCESS) return KVR_ERR_INVALID_ARG;
+        const size_t plane_bytes = (size_t)g->num_blocks * g->block_size * row_bytes;
+        const size_t end = (size_t)((uintptr_t)arena_dev - (uintptr_t)abase) + ((size_t)layer + 1) * 2 * plane_bytes;
+        if (end > asize) return KVR_ERR_INVALID_ARG;
+    }
 
     unsigned char *scratch = nullptr;
     {
@@ -100,10 +124,11 @@ extern "C" int kv_readback_noalloc(const void *arena_dev, const kv_arena_geometr
     readback_noalloc_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(plane, kv_stride_v, row_v, d_table,
                                                                             g->block_size, n, (uint4 *)d_k,
                                                                             (uint4 *)d_v);
-    if (cudaGetLastError() != cudaSuccess) return KVR_ERR_CUDA;
-    if (cudaMemcpyAsync(k_out, d_k, dense, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemcpyAsync(v_out, d_v, dense, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaStreamSynchronize(s) != cudaSuccess)
-        return KVR_ERR_CUDA;
-    return KVR_OK;
+    // From here on work may be in flight on the shared array: every return waits for the stream,
+    // so that a failed call cannot race with the next one.
+    bool ok = cudaGetLastError() == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(k_out, d_k, dense, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(v_out, d_v, dense, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    const bool synced = cudaStreamSynchronize(s) == cudaSuccess;
+    return ok && synced ? KVR_OK : KVR_ERR_CUDA;
 }

@@ -91,6 +91,30 @@ def test_lengths_around_every_boundary_wide_heads(attn):
     print("boundary lens hd128 attn", attn, worst)
 
 
+@pytest.mark.parametrize("heads", [(4, 1), (3, 1), (6, 3)])
+def test_head_layouts_that_do_not_fill_128_column_tiles(heads):
+    """Head dim 64 with q or k/v widths that are not multiples of 128 (kv_dim 64, q_dim 192): the fused
+    projection epilogue cannot split a 128-column half between q, k and v, so these shapes must take
+    the separate projection + RoPE/scatter step -- same rows, neighbouring slots and blocks untouched."""
+    hq, hkv = heads
+    shape = ModelShape("oddheads", n_layers=2, d_model=256, n_q_heads=hq, n_kv_heads=hkv, head_dim=64, ffn=512,
+                       vocab=512)
+    lens = [1, 16, 17, 130, 300]
+    batch = _batch(lens, shape.vocab, 64, 11)
+    rig = Rig(shape, "bf16", 64, max_chunk=256, max_requests=len(lens), max_blocks_per_req=batch.tables.shape[1],
+              seed=12)
+    before = rig.arena_bits()
+    rig.rebuild(batch)
+    kv = oracle_kv(weights_to_cpu(rig.weights), shape, batch)
+    worst = compare_rebuilt(rig, batch, kv, 1e-2, 6e-2)
+    check_untouched(rig, before, batch)
+    first = rig.arena_bits()
+    rig.rebuild(batch)
+    assert np.array_equal(rig.arena_bits(), first)
+    assert rig.guards_ok()
+    print("odd head layout", heads, worst)
+
+
 @pytest.mark.parametrize("chunk", [1, 7])
 def test_chunks_of_a_few_tokens(chunk):
     batch = _batch([5, 40, 18], TINY.vocab, 16, 5)

@@ -34,6 +34,27 @@ def test_health_probe_matches_oracle_and_reports_timeouts():
     assert ctx.kv_sync_status() == 0
 
 
+def test_health_probe_same_seed_twice_cannot_pass_on_stale_flags():
+    """A caller that probes with a constant seed: the flags the first call left
+    behind must not satisfy the second call's waits.  With publishing muted the
+    second call has to run out, exactly as a first call would."""
+    from paper_2608_14635_b200 import binding as kb
+    ctx = kb.Context(0)
+    n_sms = torch.cuda.get_device_properties(0).multi_processor_count
+    st, got = ctx.kv_health_probe(1, 200)
+    assert st == 0 and got == oracle.probe_checksum(1, n_sms)
+    assert ctx.kv_set_option("probe_mute", 1) == 0
+    t0 = time.perf_counter()
+    st, _ = ctx.kv_health_probe(1, 20)
+    dt = time.perf_counter() - t0
+    assert kb.STATUS[st] == "KVR_ERR_DEVICE_TIMEOUT" and dt < 2.0
+    assert ctx.kv_set_option("probe_mute", 0) == 0
+    for _ in range(3):                                   # and the same seed keeps passing unmuted
+        st, got = ctx.kv_health_probe(1, 200)
+        assert st == 0 and got == oracle.probe_checksum(1, n_sms)
+    assert ctx.kv_sync_status() == 0
+
+
 def test_flush_then_rebuild():
     shape = MODEL_SHAPES["tiny"]
     wl = make_workload(WORKLOADS["cfg1"])

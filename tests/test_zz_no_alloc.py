@@ -5,6 +5,7 @@ kv_readback returns, on two calls in a row (they share one fixed staging
 array), and refuse requests larger than that array."""
 import numpy as np
 import pytest
+import torch
 
 from synth import MODEL_SHAPES, WORKLOADS, make_workload
 from kvr_harness import Rig
@@ -21,11 +22,18 @@ def test_noalloc_readback_matches_readback_twice():
     rig.rebuild(batch)
     kb = rig.kb
     # two calls in a row, different request / layer / length: the second must not see the first's bytes
+    free_after_first = None
     for r, layer in ((3, 0), (1, 1), (3, 1)):
         n = int(batch.lens[r])
         st0, k0, v0 = rig.ctx.kv_readback(layer, batch.tables[r], n)
         st1, k1, v1 = kb.kv_readback_noalloc(rig.arena, rig.ctx.geom, layer, batch.tables[r], n)
         assert st0 == 0 and st1 == 0
+        # nothing is allocated on the device: once the first call has run (the runtime may load the
+        # library's device image lazily on it), free device memory no longer moves
+        torch.cuda.synchronize()
+        free_now = torch.cuda.mem_get_info(rig.dev)[0]
+        assert free_after_first is None or free_now == free_after_first
+        free_after_first = free_now
         assert np.array_equal(k0, k1) and np.array_equal(v0, v1)     # byte work: bit-exact
         assert not ((k1 & 0x7FFF) > 0x7F80).any()                    # rebuilt rows, not the NaN fill
     # limits: more than 2 MiB of K per call, or a bad table, is refused with a clear code
@@ -39,4 +47,9 @@ def test_noalloc_readback_matches_readback_twice():
     assert kb.STATUS[kb.kv_readback_noalloc(rig.arena, rig.ctx.geom, 0, bad, 5)[0]] == "KVR_ERR_BLOCK_OOB"
     assert kb.STATUS[kb.kv_readback_noalloc(rig.arena, rig.ctx.geom, 7, batch.tables[0], 5)[0]] == "KVR_ERR_INVALID_ARG"
     assert kb.kv_readback_noalloc(rig.arena, rig.ctx.geom, 0, batch.tables[0], 0)[0] == 0
+    # a geometry that reaches past the allocation holding the arena is refused, not read
+    import copy
+    wide = copy.copy(rig.ctx.geom)
+    wide.num_blocks = 1 << 24
+    assert kb.STATUS[kb.kv_readback_noalloc(rig.arena, wide, 1, batch.tables[0], 5)[0]] == "KVR_ERR_INVALID_ARG"
     assert rig.guards_ok()
