@@ -204,14 +204,16 @@ def resume_logits(weights: Dict[str, object], shape, tokens: np.ndarray, final_g
     return (f @ _f64(lm_head).T)[0]
 
 
-def prefill_kv_rows(weights: Dict[str, object], shape, tokens: np.ndarray, rows) -> Tuple[np.ndarray, np.ndarray,
-                                                                                          np.ndarray, np.ndarray]:
+def prefill_kv_rows(weights: Dict[str, object], shape, tokens: np.ndarray, rows,
+                    act_bf16: bool = False) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
     """Sampled outputs of a long prefix, one row at a time: layer-0 K/V of every token (they need
     no attention) and layer-1 K/V of the tokens listed in `rows` only -- for those the layer-0
     attention row is written out as its definition (scores against keys 0..t, softmax, weighted sum
     of the values), followed by the rest of layer 0 and layer 1's projections.  Same mathematics
     as prefill_kv(n_layers=2) restricted to those rows, at a cost linear in the prefix length per
-    sampled row.  Returns (K0 [n,Hkv,hd], V0 [n,Hkv,hd], K1 [len(rows),Hkv,hd], V1 [len(rows),Hkv,hd])."""
+    sampled row; `act_bf16` applies the same storage rule as there (the same eight tensors rounded
+    where they are produced).  Returns (K0 [n,Hkv,hd], V0 [n,Hkv,hd], K1 [len(rows),Hkv,hd],
+    V1 [len(rows),Hkv,hd]), unrounded."""
     tokens = np.asarray(tokens, dtype=np.int64)
     rows = np.asarray(rows, dtype=np.int64)
     n = tokens.shape[0]
@@ -223,24 +225,26 @@ def prefill_kv_rows(weights: Dict[str, object], shape, tokens: np.ndarray, rows)
         h = _f64(emb[torch.as_tensor(tokens, device=emb.device)])
     else:
         h = _f64(emb[tokens])
+    rb = round_bf16 if act_bf16 else (lambda x: x)
     w0, w1 = _layer_weights(weights, 0), _layer_weights(weights, 1)
     pos = np.arange(n)
-    q, k, v = project_qkv(rmsnorm(h, w0["ln1"], shape.rms_eps), w0, shape)
+    q, k, v = project_qkv(rb(rmsnorm(h, w0["ln1"], shape.rms_eps)), w0, shape)
     q = apply_rope(q, pos, shape.rope_base)
     k = apply_rope(k, pos, shape.rope_base)
+    qs, ks, vs = rb(q), rb(k), rb(v)          # what attention reads (k, v themselves are returned unrounded)
     K1 = np.zeros((len(rows), Hkv, hd))
     V1 = np.zeros((len(rows), Hkv, hd))
     for i, t in enumerate(rows):
         o = np.zeros((Hq, hd))
         for hq in range(Hq):
             hk = hq // G
-            sc = k[:t + 1, hk, :] @ q[t, hq, :] / math.sqrt(hd)
+            sc = ks[:t + 1, hk, :] @ qs[t, hq, :] / math.sqrt(hd)
             pr = np.exp(sc - sc.max())
-            o[hq] = (pr / pr.sum()) @ v[:t + 1, hk, :]
-        x = h[t] + w0["wo"] @ o.reshape(-1)
-        b = rmsnorm(x[None], w0["ln2"], shape.rms_eps)[0]
-        x = x + w0["wd"] @ (silu(w0["wg"] @ b) * (w0["wu"] @ b))
-        a1 = rmsnorm(x[None], w1["ln1"], shape.rms_eps)
+            o[hq] = (rb(pr) @ vs[:t + 1, hk, :]) / pr.sum()
+        x = h[t] + w0["wo"] @ rb(o).reshape(-1)
+        b = rb(rmsnorm(x[None], w0["ln2"], shape.rms_eps)[0])
+        x = x + w0["wd"] @ rb(silu(w0["wg"] @ b) * (w0["wu"] @ b))
+        a1 = rb(rmsnorm(x[None], w1["ln1"], shape.rms_eps))
         _, k1, v1 = project_qkv(a1, w1, shape)
         K1[i] = apply_rope(k1, np.array([t]), shape.rope_base)[0]
         V1[i] = v1[0]

@@ -350,3 +350,9 @@ def test_sampled_rows_equal_the_full_prefill():
         assert rel(K0, K[0]) < 1e-13 and rel(V0, V[0]) < 1e-13
         assert rel(K1, K[1][rows]) < 1e-12 and rel(V1, V[1][rows]) < 1e-12
         assert rel(K1, K[1][[r + 1 for r in rows[:-1]] + [0]]) > 1e-2      # the rows are not interchangeable
+        # the bf16 storage reading, row by row, is the full prefill's
+        Kf, Vf = oracle.prefill_kv(w, shape, toks, n_layers=2, act_bf16=True)
+        K0f, V0f, K1f, V1f = oracle.prefill_kv_rows(w, shape, toks, rows, act_bf16=True)
+        assert rel(K0f, Kf[0]) < 1e-13 and rel(V0f, Vf[0]) < 1e-13
+        assert rel(K1f, Kf[1][rows]) < 1e-12 and rel(V1f, Vf[1][rows]) < 1e-12
+        assert 1e-4 < rel(K1f, K1) < 3e-2                                  # and it does differ from the definition
