@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _free_device_memory_after_each_test():
+    """A failed test's traceback keeps its frame alive; the tens of GB a full-size rig holds must
+    not stay allocated for the tests that follow."""
+    yield
+    import sys
+    harness = sys.modules.get("kvr_harness")
+    if harness is not None:
+        harness.free_live()

@@ -7,11 +7,12 @@ long request (layer l's K/V depend only on layers < l).  Everything else is
 covered by properties that hold at any size: untouched bytes bit-exact,
 idempotence bit-exact, no fill left in a mapped row.
 
-Tolerance at depth.  rel-L2 <= 1e-2 / max-abs <= 6e-2 is asserted outright on
-the first two layers.  Deeper, the bf16 storage of activations alone (the
-oracle's own forward with exact arithmetic but bf16-rounded activation
-tensors) drifts past 1e-2 on these random-init shapes; there the GPU result is
-required to stay within 15 % of that format floor (see compare_readback)."""
+Tolerance at depth.  Expected values always come from the oracle's definition.
+rel-L2 <= 1e-2 / max-abs <= 6e-2 is asserted wherever the bf16 format itself can
+meet it.  Deeper, the bf16 storage of activations alone (the oracle's own forward
+with exact arithmetic but bf16-rounded activation tensors) drifts past it on
+these random-init shapes; there the GPU result must stay within a few per cent of
+that format floor (margins and the per-layer table: see compare_readback)."""
 import dataclasses
 
 import numpy as np
@@ -20,7 +21,8 @@ import torch
 
 import oracle
 from synth import MODEL_SHAPES, WORKLOADS, BENCH_CHUNK_TOKENS, make_workload
-from kvr_harness import Rig, weights_to_cpu, compare_readback, check_untouched_on_device
+from kvr_harness import (Rig, weights_to_cpu, compare_readback, check_untouched_on_device, oracle_weights,
+                         oracle_definition_and_floor)
 
 pytestmark = pytest.mark.gpu
 BF16_REL, BF16_ABS = 1e-2, 6e-2
@@ -53,14 +55,13 @@ def test_cfg2_full_batch_sampled_parity():
         assert np.array_equal(slots[off[r]:off[r + 1]], batch.tables[r][t // 16].astype(np.int64) * 16 + t % 16)
     check_untouched_on_device(rig, batch)
     # full depth: the two shortest requests whole, 384-token truncations of the longest and one more
-    w_cpu = weights_to_cpu(rig.weights)
+    w_cpu = oracle_weights(rig.weights)
     order = np.argsort(batch.lens)
     picks = {int(order[0]): int(batch.lens[order[0]]), int(order[1]): min(int(batch.lens[order[1]]), 640),
              int(order[-1]): 384, int(order[len(order) // 2]): 384}
     kv, floor = {}, {}
     for r, n in picks.items():
-        kv[r] = oracle.prefill_kv(w_cpu, shape, batch.tokens[off[r]:off[r] + n])
-        floor[r] = oracle.prefill_kv(w_cpu, shape, batch.tokens[off[r]:off[r] + n], act_bf16=True)
+        kv[r], floor[r] = oracle_definition_and_floor(w_cpu, shape, batch.tokens[off[r]:off[r] + n])
     worst = compare_readback(rig, batch, kv, BF16_REL, BF16_ABS, kv_format_floor=floor, label="cfg2")
     print("cfg2 full-depth sampled worst", worst, "picks", picks)
     # idempotence at full size, bit for bit (compared on the device)
@@ -101,12 +102,11 @@ def test_cfg3_full_batch_sampled_parity():
     rig.rebuild(batch)
     check_untouched_on_device(rig, batch)
     off = np.concatenate([[0], np.cumsum(batch.lens)])
-    w_cpu = weights_to_cpu(rig.weights)
+    w_cpu = oracle_weights(rig.weights)
     order = np.argsort(batch.lens)
     kv, floor = {}, {}
     for r in (int(order[0]), int(order[-1])):
-        kv[r] = oracle.prefill_kv(w_cpu, shape, batch.tokens[off[r]:off[r] + 256])
-        floor[r] = oracle.prefill_kv(w_cpu, shape, batch.tokens[off[r]:off[r] + 256], act_bf16=True)
+        kv[r], floor[r] = oracle_definition_and_floor(w_cpu, shape, batch.tokens[off[r]:off[r] + 256])
     worst = compare_readback(rig, batch, kv, BF16_REL, BF16_ABS, kv_format_floor=floor, label="cfg3")
     print("cfg3 full-depth sampled worst", worst)
     assert rig.guards_ok()
