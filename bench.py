@@ -427,8 +427,8 @@ def main():
                     help="optional projection terms: q/k/v biases or per-head q/k RMSNorm (default: the headline model)")
     ap.add_argument("--gemm", type=int, default=None, choices=[1, 2],
                     help="tcgen05 GEMM tiling: 1 = single-CTA 128x256 tiles, 2 = CTA pairs (default: the library's)")
-    ap.add_argument("--attn", type=int, default=None, choices=[1, 2, 3],
-                    help="attention kernel: 1 = warp MMA, 2 = tcgen05 single CTA, 3 = tcgen05 CTA pairs (default: the library's)")
+    ap.add_argument("--attn", type=int, default=None, choices=[1, 2],
+                    help="attention kernel: 1 = warp MMA, 2 = tcgen05 (default: the library's)")
     ap.add_argument("--layers", type=int, default=None, help="profiling aid: run only this many layers")
     ap.add_argument("--requests", type=int, default=None, help="profiling aid: rebuild only the first N requests")
     args = ap.parse_args()

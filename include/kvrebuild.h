@@ -277,11 +277,13 @@ int kv_debug_plan(kvr_ctx *ctx, int64_t *computed_tokens, int64_t *n_chunks, int
 int kv_debug_profile(kvr_ctx *ctx, double *ms_by_kind, int64_t *launches_by_kind);
 
 /* Options: "keep_last_hidden" 0/1 (see kv_resume_logits; default 0); "probe_mute" 0/1 (test hook: probe blocks do not publish their flags, so every
- * device wait of kv_health_probe runs out; default 0); "profile" 0/1 (see kv_debug_profile; default 0); "gemm" 0 = plain-FMA kernels,
+ * device wait of kv_health_probe runs out; default 0); "wait_limit_ms" 0..60000 (how long a wait inside the tensor-core GEMM and attention
+ * kernels may last before the kernel gives up, records KVR_ERR_DEVICE_TIMEOUT for kv_sync_status and returns; 0 = the default of about 2 s);
+ * "mute_loads" 0/1 (test hook: the TMA producers of those kernels issue no loads, so every wait on their data runs out and nothing is
+ * written; default 0); "profile" 0/1 (see kv_debug_profile; default 0); "gemm" 0 = plain-FMA kernels,
  * 1 = tcgen05 kernels on 128 x 256 tiles, 2 = tcgen05 kernels on CTA pairs (256 x 256 tiles); 1 and 2 are bf16 only, 2 is the default in bf16;
- * "attn" 0 = plain kernel, 1 = warp-level MMA kernel, 2 = tcgen05 kernel, 3 = tcgen05 kernel on
- * CTA pairs (1-3 bf16 only; 2 is the default in bf16; 2 and 3 need block_size 16, 3 also head_dim 128,
- * otherwise the next lower one is used).
+ * "attn" 0 = plain kernel, 1 = warp-level MMA kernel, 2 = tcgen05 kernel (1 and 2 bf16 only; 2 is the
+ * default in bf16 and needs block_size 16, otherwise 1 is used).
  * Returns KVR_ERR_INVALID_ARG for unknown names or values. */
 int kv_set_option(kvr_ctx *ctx, const char *name, int64_t value);
 

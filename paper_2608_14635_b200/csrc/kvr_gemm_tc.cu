@@ -374,7 +374,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int num_k = (ep.K + BK - 1) / BK;
 
     if (warp == 0) {
-        if (lane == 0) {
+        if (lane == 0 && !ptx::loads_muted(status)) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -525,7 +525,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int num_k = (ep.K + BK - 1) / BK;
 
     if (warp == 0) {
-        if (lane == 0) {
+        if (lane == 0 && !ptx::loads_muted(status)) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;

@@ -19,7 +19,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct WsLayout {
     size_t h, a, q, m, cs, meta, tables, tiles, total;
-    size_t l_h, l_a, l_q, l_m, l_cs, l_pos, l_pairs, l_tiles;   // per-request buffers for kv_resume_logits
+    size_t l_h, l_a, l_q, l_m, l_cs, l_pos, l_pairs, l_tiles, l_part;   // per-request buffers for kv_resume_logits
     size_t m_bytes;
 };
 
@@ -34,7 +34,9 @@ struct Chunk {
 struct kvr_ctx {
     int device = 0;
     int n_sms = 0;
-    int *d_status = nullptr;
+    int *d_status = nullptr;       // device status block: [0] status, [1] flags, [2..3] wait limit in cycles
+    int wait_limit_ms = 0;         // 0 = the default of about two seconds
+    int mute_loads = 0;
     // arena
     bool arena_bound = false;
     kv_arena_geometry geom{};
@@ -55,7 +57,7 @@ struct kvr_ctx {
     int64_t max_chunk = 0;
     int32_t max_req = 0, max_blk = 0;
     WsLayout lay{};
-    CUtensorMap tm_a_d{}, tm_a_q{}, tm_m{}, tm_q{}, tm_kv{}, tm_kv2{}, tm_h{};
+    CUtensorMap tm_a_d{}, tm_a_q{}, tm_m{}, tm_q{}, tm_kv{}, tm_h{};
     bool tm_kv_ok = false;
     // pinned staging
     char *pinned = nullptr;
@@ -84,6 +86,17 @@ struct kvr_ctx {
 namespace {
 
 enum { W_LN1 = 0, W_WQ, W_WK, W_WV, W_WO, W_LN2, W_WG, W_WU, W_WD };
+
+// Flags and wait limit of the device status block (the status word itself is left alone).
+static int write_status_block(kvr_ctx *c) {
+    const long long ms = c->wait_limit_ms > 0 ? c->wait_limit_ms : 2000;
+    int32_t words[3];
+    const long long cycles = ms * (long long)std::max(c->clock_khz, 1000);
+    words[0] = c->mute_loads ? 1 : 0;
+    std::memcpy(&words[1], &cycles, sizeof(cycles));
+    return cudaMemcpy(c->d_status + 1, words, sizeof(words), cudaMemcpyHostToDevice) == cudaSuccess ? KVR_OK
+                                                                                                     : KVR_ERR_CUDA;
+}
 
 // optional projection terms of layer l (null pointers where the bound set has none)
 static QkvExtras qkv_extras(const kvr_ctx *c, int l) {
@@ -130,6 +143,7 @@ bool compute_layout(const kvr_ctx *c, int64_t Tc, int32_t max_req, int32_t max_b
     L->l_pos = o; o += align_up(Rq * 2 * sizeof(int32_t));
     L->l_pairs = o; o += align_up(Rq * sizeof(int2));
     L->l_tiles = o; o += align_up(Rq * sizeof(AttnTile));
+    L->l_part = o; o += align_up(attn_decode_scratch_bytes(max_req, md.Hq, md.hd));
     L->total = o;
     return true;
 }
@@ -337,16 +351,16 @@ int kv_ctx_create(kvr_ctx **out, int device) {
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return KVR_ERR_CUDA; }
     c->n_sms = prop.multiProcessorCount;
     cudaDeviceGetAttribute(&c->clock_khz, cudaDevAttrClockRate, device);
-    if (cudaMalloc((void **)&c->d_status, sizeof(int)) != cudaSuccess ||
+    if (cudaMalloc((void **)&c->d_status, 4 * sizeof(int)) != cudaSuccess ||
         cudaMalloc((void **)&c->d_probe, 2 * PROBE_MAX_BLOCKS * sizeof(uint32_t)) != cudaSuccess ||
         cudaMemset(c->d_probe, 0, 2 * PROBE_MAX_BLOCKS * sizeof(uint32_t)) != cudaSuccess ||
-        cudaMemset(c->d_status, 0, sizeof(int)) != cudaSuccess ||
+        cudaMemset(c->d_status, 0, 4 * sizeof(int)) != cudaSuccess || write_status_block(c) != KVR_OK ||
         cudaEventCreateWithFlags(&c->staging_free, cudaEventDisableTiming) != cudaSuccess) {
         delete c;
         return KVR_ERR_CUDA;
     }
     c->tc_ready = (prop.major == 10) && tc_gemm_init(device) == KVR_OK && attn_tc_init(device) == KVR_OK &&
-                  attn_fa_init(device) == KVR_OK && attn_fa2_init(device) == KVR_OK;
+                  attn_fa_init(device) == KVR_OK;
     *out = c;
     return KVR_OK;
 }
@@ -396,8 +410,7 @@ int kv_arena_bind(kvr_ctx *c, void *arena, size_t bytes, const kv_arena_geometry
         (g->head_dim == 64 || g->head_dim == 128)) {
         const int64_t rows2d = (int64_t)g->n_layers * 2 * slots;
         if (rows2d < ((int64_t)1 << 31) &&
-            tc_make_tmap_kv(&c->tm_kv, arena, rows2d, row, g->head_dim / 64) == KVR_OK &&
-            tc_make_tmap_2d(&c->tm_kv2, arena, rows2d, row, 16, 64) == KVR_OK)
+            tc_make_tmap_kv(&c->tm_kv, arena, rows2d, row, g->head_dim / 64) == KVR_OK)
             c->tm_kv_ok = true;
     }
     c->arena_bound = true;
@@ -516,7 +529,7 @@ int kv_workspace_bind(kvr_ctx *c, void *ws, size_t bytes, int64_t max_chunk_toke
 int kv_set_option(kvr_ctx *c, const char *name, int64_t value) {
     if (!c || !name) return KVR_ERR_INVALID_ARG;
     if (!std::strcmp(name, "attn")) {
-        if (value < 0 || value > 3) return KVR_ERR_INVALID_ARG;
+        if (value < 0 || value > 2) return KVR_ERR_INVALID_ARG;
         c->attn_impl = (int)value;
         return KVR_OK;
     }
@@ -525,7 +538,18 @@ int kv_set_option(kvr_ctx *c, const char *name, int64_t value) {
         c->gemm_impl = (int)value;
         return KVR_OK;
     }
+    if (!std::strcmp(name, "wait_limit_ms")) {
+        if (value < 0 || value > 60000) return KVR_ERR_INVALID_ARG;
+        SetDevice sd(c->device);
+        c->wait_limit_ms = (int)value;
+        return write_status_block(c);
+    }
     if (value != 0 && value != 1) return KVR_ERR_INVALID_ARG;
+    if (!std::strcmp(name, "mute_loads")) {
+        SetDevice sd(c->device);
+        c->mute_loads = (int)value;
+        return write_status_block(c);
+    }
     if (!std::strcmp(name, "profile")) { c->profile = (int)value; return KVR_OK; }
     if (!std::strcmp(name, "probe_mute")) { c->probe_mute = (int)value; return KVR_OK; }
     if (!std::strcmp(name, "keep_last_hidden")) { c->keep_last = (int)value; return KVR_OK; }
@@ -556,9 +580,8 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     // q_dim and kv_dim to be multiples of 128; other head counts take the plain projection + RoPE/scatter
     // kernels for this one step (same arena rows, no tile ever straddles two destinations).
     const bool use_tc_qkv = use_tc_gemm && md.q_dim % 128 == 0 && md.kv_dim % 128 == 0;
-    // tcgen05 attention needs 16-slot blocks (the CTA-pair kernel also head dim 128): the next kernel down takes over
-    const bool use_fa2_attn = !fp32 && c->attn_impl == 3 && c->tm_kv_ok && md.hd == 128;
-    const bool use_fa_attn = !fp32 && c->attn_impl >= 2 && c->tm_kv_ok;   // either tcgen05 kernel
+    // tcgen05 attention needs 16-slot blocks: otherwise the warp-MMA kernel takes over
+    const bool use_fa_attn = !fp32 && c->attn_impl >= 2 && c->tm_kv_ok;
     const bool use_tc_attn = !fp32 && (c->attn_impl == 1 || (c->attn_impl >= 2 && !use_fa_attn));
     const int tile_q = use_fa_attn ? ATTN_FA_TILE_Q : ATTN_TILE_Q;
     if ((use_tc_gemm || use_tc_attn || use_fa_attn) && !c->tc_ready) return KVR_ERR_UNSUPPORTED;
@@ -737,11 +760,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
             // causal attention over the paged K/V just written (output into `a`)
             {
                 Timed tm(c, 4, s);
-                if (use_fa2_attn) {
-                    st = launch_attn_fa2(c->tm_q, c->tm_kv, c->tm_kv2, d_tiles, n_tiles, d_tables, width, md, c->av, l,
-                                         (__nv_bfloat16 *)a, c->d_status, s);
-                    if (st != KVR_OK) return st;
-                } else if (use_fa_attn) {
+                if (use_fa_attn) {
                     st = launch_attn_fa(c->tm_q, c->tm_kv, d_tiles, n_tiles, d_tables, width, md, c->av, l,
                                         (__nv_bfloat16 *)a, c->d_status, s);
                     if (st != KVR_OK) return st;
@@ -939,7 +958,15 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         q_only.Hkv = 0; q_only.kv_dim = 0;
         launch_rope_scatter(fp32, tmp, md.q_dim, cs, cm, q_only, c->av, l, true, q, ex, s);
     }
-    if (use_fa) {
+    // one query row per request: the split-KV kernel reads each request's K/V once (bf16, groups of up to 8 heads)
+    const bool use_decode = !fp32 && c->attn_impl != 0 && md.Hq / md.Hkv <= 8;
+    if (use_decode) {
+        int max_len = 0;
+        for (int r = 0; r < R; ++r) max_len = std::max(max_len, c->last_lens[r]);
+        st = launch_attn_decode((const __nv_bfloat16 *)q, d_pos, R, max_len, d_tables, width, md, c->av, l,
+                                (float *)(ws + L.l_part), (__nv_bfloat16 *)a, s);
+        if (st != KVR_OK) return st;
+    } else if (use_fa) {
         st = launch_attn_fa(c->tm_lq, c->tm_kv, d_tiles, R, d_tables, width, md, c->av, l, (__nv_bfloat16 *)a,
                             c->d_status, s);
         if (st != KVR_OK) return st;

@@ -118,19 +118,20 @@ int launch_attn_tc(const __nv_bfloat16 *q, const AttnTile *tiles, int n_tiles, c
                    cudaStream_t s);
 constexpr int ATTN_TILE_Q = 64;
 
-// ---- tcgen05 attention on CTA pairs (kvr_attn_fa2.cu): head dim 128, tiles of up to 256 query rows ----
-// tmK: 4-D block map (tc_make_tmap_kv), tmV: 2-D map with 16-row x 64-column boxes.
-int attn_fa2_init(int device);
-int launch_attn_fa2(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const AttnTile *tiles,
-                    int n_tiles, const int32_t *tables, int max_blk, const ModelDims &md, const ArenaView &av,
-                    int layer, __nv_bfloat16 *o, int *d_status, cudaStream_t s);
-
 // ---- tcgen05 attention (kvr_attn_fa.cu): tiles of up to 256 query rows ----
 constexpr int ATTN_FA_TILE_Q = 256;
 int attn_fa_init(int device);
 int launch_attn_fa(const CUtensorMap &tmQ, const CUtensorMap &tmKV, const AttnTile *tiles, int n_tiles,
                    const int32_t *tables, int max_blk, const ModelDims &md, const ArenaView &av, int layer,
                    __nv_bfloat16 *o, int *d_status, cudaStream_t s);
+
+// ---- single-row attention for resume logits (kvr_attn_decode.cu): split-KV, one pass over the request's K/V ----
+constexpr int ATTN_DECODE_MAX_SPLITS = 16;
+size_t attn_decode_scratch_bytes(int max_requests, int Hq, int hd);
+// q [R, Hq*hd] bf16, pos[r] = position of the query row (it attends to keys 0..pos[r]); max_len = max(pos) + 1
+int launch_attn_decode(const __nv_bfloat16 *q, const int32_t *pos, int R, int max_len, const int32_t *tables,
+                       int max_blk, const ModelDims &md, const ArenaView &av, int layer, float *scratch,
+                       __nv_bfloat16 *o, cudaStream_t s);
 
 // ---- handover device steps (kvr_handover.cu) ----
 constexpr int PROBE_THREADS = 64, PROBE_ITERS = 1000, PROBE_MAX_BLOCKS = 1024;

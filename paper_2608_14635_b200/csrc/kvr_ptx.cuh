@@ -40,17 +40,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Wait for a phase with a cycle limit.  Returns false (and records the
-// failure in *status) if the limit expires, so that no wait can hang the GPU.
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // about two seconds
+// Device status block of a context (four 32-bit words, 8-byte aligned):
+//   [0] status word: 0, or a kvr_status a kernel recorded (a wait that ran out)
+//   [1] flags, bit 0: test hook, TMA producers issue no loads (every wait on their data runs out)
+//   [2..3] limit of a device-side wait in SM cycles (64-bit)
+constexpr int STATUS_FLAGS = 1, STATUS_LIMIT = 2;
+constexpr uint32_t FLAG_MUTE_LOADS = 1u;
+__device__ __forceinline__ bool loads_muted(const int *status) {
+    return (*reinterpret_cast<const volatile uint32_t *>(status + STATUS_FLAGS) & FLAG_MUTE_LOADS) != 0;
+}
+// Wait for a phase with a cycle limit (read from the status block, only once the
+// first probe has failed).  Returns false (and records the failure in *status)
+// if the limit expires, so that no wait can hang the GPU.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *status, volatile int *abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
+    const long long limit = *reinterpret_cast<const volatile long long *>(status + STATUS_LIMIT);
     const long long t0 = clock64();
     while (true) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             atomicExch(status, -10);
             return false;

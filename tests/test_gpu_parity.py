@@ -229,7 +229,7 @@ def test_gemm_kernels_against_fp64(M, N, K):
         assert err < tol, (impl, err)
 
 
-@pytest.mark.parametrize("attn", [1, 2, 3])
+@pytest.mark.parametrize("attn", [1, 2])
 def test_mid_shape_bf16_parity(attn):
     """A mid-size decoder (hd 128, GQA group 4, ffn not a multiple of 256) with
     lengths that span several tiles, a ragged tail and a chunk boundary."""
