@@ -112,6 +112,45 @@ typedef struct {
 } kv_proj_variant;
 int kv_variant_bind(kvr_ctx *ctx, const kv_proj_variant *variant);
 
+/* Paper Sec. 6.1 (experimental setup): the rollout engines whose KV is rebuilt are tensor-parallel
+ * (TP = 2 / 4).  Under TP every rank holds the whole residual stream, its own share of the
+ * attention heads and of the SwiGLU columns, and its own KV pool with its share of the kv heads;
+ * the two row-parallel products of a layer (output projection, down projection) yield partial
+ * sums that are added over the ranks before they enter the residual.
+ *
+ * A context runs one rank.  The shapes it is bound with are the rank's LOCAL ones
+ * (kv_tp_plan_host gives them): n_q_heads, n_kv_heads and ffn are per-rank counts, d_model and
+ * vocab are whole; weights are the rank's slices (wq/wk/wv/wg/wu: a range of rows, wo/wd: a range
+ * of columns, as contiguous matrices of the local shape; norms and embedding whole); the arena is
+ * the rank's pool (n_kv_heads local).  kv_tp_bind then names the exchange step:
+ *   allreduce(buf_dev, count, stream, user) must enqueue on `stream` an in-place sum over all
+ *   ranks of `count` fp32 values at buf_dev (device memory of this rank) and return 0, or return
+ *   non-zero on failure (kv_rebuild then returns KVR_ERR_CUDA).  It is called on the host, inside
+ *   kv_rebuild, twice per layer and chunk, in the same order on every rank; the library itself
+ *   contains no collective and never touches another rank's memory.
+ * tp_world = 1 (or config NULL) clears the sharding.  Call after kv_weights_bind and before
+ * kv_workspace_bytes / kv_workspace_bind (the workspace gains one fp32 [chunk, d_model] buffer).
+ * All ranks must be given the same batch, chunk size and options.  kv_resume_logits is not
+ * available under TP (KVR_ERR_UNSUPPORTED). */
+typedef int (*kv_allreduce_fn)(void *buf_dev, int64_t count, void *stream, void *user);
+typedef struct {
+    int32_t tp_world, tp_rank;
+    kv_allreduce_fn allreduce;
+    void *user;
+} kv_tp_config;
+int kv_tp_bind(kvr_ctx *ctx, const kv_tp_config *config);
+
+/* Host-only partition plan of a model over tp_world ranks (needs no GPU and no context): rank r
+ * takes q heads [q_head0, q_head0 + n_q_heads), kv heads [kv_head0, ...) -- whole GQA groups, so a
+ * rank's q heads only ever read its own kv heads -- and SwiGLU columns [ffn0, ffn0 + ffn).
+ * local_out receives the descriptor to bind on that rank.  KVR_ERR_UNSUPPORTED if tp_world does
+ * not divide n_kv_heads and ffn / 8. */
+typedef struct {
+    int32_t q_head0, n_q_heads, kv_head0, n_kv_heads, ffn0, ffn;
+} kv_tp_shard;
+int kv_tp_plan_host(const kv_model_desc *full, int32_t tp_world, int32_t tp_rank, kv_model_desc *local_out,
+                    kv_tp_shard *shard_out);
+
 /* Scratch the rebuild needs for chunks of at most max_chunk_tokens tokens,
  * batches of at most max_requests requests and tables of at most
  * max_blocks_per_req entries.  Needs the weights bound (for the shape).

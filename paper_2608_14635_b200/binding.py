@@ -27,7 +27,7 @@ EXPORTS = ("kv_ctx_create", "kv_ctx_destroy", "kv_arena_bind", "kv_weights_bind"
            "kv_workspace_bind", "kv_rebuild", "kv_readback", "kv_readback_dev", "kv_sync_status",
            "kv_check_inputs", "kv_debug_slot_map", "kv_debug_plan", "kv_debug_profile", "kv_set_option", "kv_debug_gemm",
            "kv_status_str", "kv_readback_noalloc", "kv_arena_flush", "kv_health_probe", "kv_resume_logits", "kv_rebuild_from",
-           "kv_variant_bind", "kv_plan_host")
+           "kv_variant_bind", "kv_plan_host", "kv_tp_bind", "kv_tp_plan_host")
 
 
 class kv_model_desc(C.Structure):
@@ -48,6 +48,17 @@ class kv_weights(C.Structure):
 
 class kv_proj_variant(C.Structure):
     _fields_ = [(n, _PP) for n in ("bq", "bk", "bv", "q_norm", "k_norm")]
+
+
+ALLREDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p)
+
+
+class kv_tp_config(C.Structure):
+    _fields_ = [("tp_world", C.c_int32), ("tp_rank", C.c_int32), ("allreduce", ALLREDUCE_FN), ("user", C.c_void_p)]
+
+
+class kv_tp_shard(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("q_head0", "n_q_heads", "kv_head0", "n_kv_heads", "ffn0", "ffn")]
 
 
 class KvrError(RuntimeError):
@@ -89,6 +100,9 @@ def _load() -> C.CDLL:
         "kv_resume_logits": (C.c_int, [vp, vp, vp, vp, vp]),
         "kv_health_probe": (C.c_int, [vp, C.c_uint32, i32, C.POINTER(C.c_uint32), vp]),
         "kv_readback_noalloc": (C.c_int, [vp, C.POINTER(kv_arena_geometry), i32, ip, i32, vp, vp, vp]),
+        "kv_tp_bind": (C.c_int, [vp, C.POINTER(kv_tp_config)]),
+        "kv_tp_plan_host": (C.c_int, [C.POINTER(kv_model_desc), i32, i32, C.POINTER(kv_model_desc),
+                                      C.POINTER(kv_tp_shard)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -136,6 +150,14 @@ def kv_plan_host(lens, tables, block_size: int, chunk_tokens: int, tile_rows: in
                           int(keep_last_hidden), chunk_tokens, tile_rows, _ip(skip), C.byref(computed),
                           C.byref(chunks), C.byref(tiles))
     return st, skip, computed.value, chunks.value, tiles.value
+
+
+def kv_tp_plan_host(shape, dtype: int, tp_world: int, tp_rank: int):
+    """Host-only partition plan -> (status, local kv_model_desc, kv_tp_shard)."""
+    full = make_desc(shape, dtype)
+    local, shard = kv_model_desc(), kv_tp_shard()
+    st = lib.kv_tp_plan_host(C.byref(full), tp_world, tp_rank, C.byref(local), C.byref(shard))
+    return st, local, shard
 
 
 def kv_readback_noalloc(arena, geom: kv_arena_geometry, layer: int, table, n_tokens: int, stream=None):
@@ -223,6 +245,19 @@ class Context:
         st = lib.kv_variant_bind(self._h, C.byref(v))
         if st == KVR_OK:
             self._keep["variant"] = weights
+        return st
+
+    def kv_tp_bind(self, tp_world: int, tp_rank: int, allreduce) -> int:
+        """`allreduce(buf_ptr, count, stream_ptr, user) -> int` is a Python callable (or None with
+        tp_world 1): it must enqueue an in-place fp32 sum over the ranks on the given stream."""
+        if tp_world <= 1:
+            self._keep.pop("tp_cb", None)
+            return lib.kv_tp_bind(self._h, None)
+        cb = ALLREDUCE_FN(allreduce)
+        cfg = kv_tp_config(tp_world, tp_rank, cb, None)
+        st = lib.kv_tp_bind(self._h, C.byref(cfg))
+        if st == KVR_OK:
+            self._keep["tp_cb"] = cb          # the library keeps the function pointer
         return st
 
     def kv_workspace_bytes(self, max_chunk_tokens: int, max_requests: int, max_blocks_per_req: int) -> int:

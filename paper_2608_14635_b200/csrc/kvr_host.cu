@@ -18,7 +18,7 @@ constexpr size_t ALIGN = 256;
 inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct WsLayout {
-    size_t h, a, q, m, cs, meta, tables, tiles, total;
+    size_t h, a, q, m, cs, meta, tables, tiles, part, total;
     size_t l_h, l_a, l_q, l_m, l_cs, l_pos, l_pairs, l_tiles, l_part;   // per-request buffers for kv_resume_logits
     size_t m_bytes;
 };
@@ -64,6 +64,10 @@ struct kvr_ctx {
     size_t pinned_bytes = 0;
     cudaEvent_t staging_free = nullptr;
     bool staging_busy = false;
+    // tensor-parallel rank (tp_world 1 = unsharded)
+    int tp_world = 1, tp_rank = 0;
+    kv_allreduce_fn tp_allreduce = nullptr;
+    void *tp_user = nullptr;
     // options
     int gemm_impl = 2, attn_impl = 2, profile = 0, probe_mute = 0;
     uint32_t *d_probe = nullptr;   // [2 * PROBE_MAX_BLOCKS]: flags, results
@@ -144,6 +148,8 @@ bool compute_layout(const kvr_ctx *c, int64_t Tc, int32_t max_req, int32_t max_b
     L->l_pairs = o; o += align_up(Rq * sizeof(int2));
     L->l_tiles = o; o += align_up(Rq * sizeof(AttnTile));
     L->l_part = o; o += align_up(attn_decode_scratch_bytes(max_req, md.Hq, md.hd));
+    L->part = o;
+    if (c->tp_world > 1) o += align_up(T * md.d * sizeof(float));   // partial sums awaiting the all-reduce
     L->total = o;
     return true;
 }
@@ -485,6 +491,45 @@ int kv_variant_bind(kvr_ctx *c, const kv_proj_variant *v) {
     return KVR_OK;
 }
 
+int kv_tp_plan_host(const kv_model_desc *full, int32_t tp_world, int32_t tp_rank, kv_model_desc *local_out,
+                    kv_tp_shard *shard_out) {
+    if (!full || tp_world < 1 || tp_rank < 0 || tp_rank >= tp_world) return KVR_ERR_INVALID_ARG;
+    if (full->n_q_heads <= 0 || full->n_kv_heads <= 0 || full->ffn <= 0 || full->n_q_heads % full->n_kv_heads)
+        return KVR_ERR_INVALID_ARG;
+    if (full->n_kv_heads % tp_world || full->ffn % (8 * tp_world)) return KVR_ERR_UNSUPPORTED;
+    const int G = full->n_q_heads / full->n_kv_heads;
+    kv_tp_shard sh;
+    sh.n_kv_heads = full->n_kv_heads / tp_world;
+    sh.kv_head0 = tp_rank * sh.n_kv_heads;
+    sh.n_q_heads = sh.n_kv_heads * G;            // whole GQA groups: a rank's q heads read only its kv heads
+    sh.q_head0 = sh.kv_head0 * G;
+    sh.ffn = full->ffn / tp_world;
+    sh.ffn0 = tp_rank * sh.ffn;
+    if (shard_out) *shard_out = sh;
+    if (local_out) {
+        *local_out = *full;
+        local_out->n_q_heads = sh.n_q_heads;
+        local_out->n_kv_heads = sh.n_kv_heads;
+        local_out->ffn = sh.ffn;
+    }
+    return KVR_OK;
+}
+
+int kv_tp_bind(kvr_ctx *c, const kv_tp_config *cfg) {
+    if (!c) return KVR_ERR_INVALID_ARG;
+    if (!c->weights_bound) return KVR_ERR_NOT_BOUND;
+    if (!cfg || cfg->tp_world <= 1) {
+        if (cfg && cfg->tp_world < 1) return KVR_ERR_INVALID_ARG;
+        c->tp_world = 1; c->tp_rank = 0; c->tp_allreduce = nullptr; c->tp_user = nullptr;
+    } else {
+        if (cfg->tp_rank < 0 || cfg->tp_rank >= cfg->tp_world || !cfg->allreduce) return KVR_ERR_INVALID_ARG;
+        c->tp_world = cfg->tp_world; c->tp_rank = cfg->tp_rank;
+        c->tp_allreduce = cfg->allreduce; c->tp_user = cfg->user;
+    }
+    c->ws_bound = false;   // the layout depends on it
+    return KVR_OK;
+}
+
 size_t kv_workspace_bytes(const kvr_ctx *c, int64_t max_chunk_tokens, int32_t max_requests,
                           int32_t max_blocks_per_req) {
     WsLayout L;
@@ -705,12 +750,22 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
         if (np > 0)
             CU_OK(cudaMemcpyAsync(d_pairs, st_pairs + pair_begin[k], (size_t)np * sizeof(int2), cudaMemcpyHostToDevice, s));
         { Timed tm(c, 0, s); launch_rope_table(cm.pos, n, md.hd, rf, cs, s); } ++launches;
+        // Tensor-parallel ranks: a row-parallel projection leaves a partial sum in `part`; once summed over
+        // the ranks it is added to the residual by the norm kernel that follows (tp_pending: still to be added).
+        const bool tp = c->tp_world > 1;
+        float *part = (float *)(ws + L.part);
+        bool tp_pending = false;
+        auto tp_allreduce = [&]() -> int {
+            return c->tp_allreduce(part, (int64_t)n * md.d, (void *)s, c->tp_user) == 0 ? KVR_OK : KVR_ERR_CUDA;
+        };
         for (int l = 0; l < md.L; ++l) {
             const bool last = (l == md.L - 1);
             {
                 Timed tm(c, l == 0 ? 1 : 2, s);
                 if (l == 0) launch_embed_rmsnorm(fp32, c->embed, c->w[W_LN1][0], cm, h, a, md.d, md.eps, s);
+                else if (tp_pending) launch_add_rmsnorm(fp32, h, part, c->w[W_LN1][l], a, n, md.d, md.eps, s);
                 else launch_rmsnorm(fp32, h, c->w[W_LN1][l], a, n, md.d, md.eps, s);
+                tp_pending = false;
             }
             ++launches;
             if (last && np > 0) {   // h entering the last layer, for the tokens that end a request
@@ -776,18 +831,27 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
             // output projection + residual
             if (use_tc_gemm) {
                 TcGemmEpilogue ep{};
-                ep.mode = TC_RESID; ep.M = n; ep.N = md.d; ep.K = md.q_dim; ep.c_f32 = h; ep.ldc = md.d;
+                ep.mode = tp ? TC_STORE_F32 : TC_RESID; ep.M = n; ep.N = md.d; ep.K = md.q_dim;
+                ep.c_f32 = tp ? part : h; ep.ldc = md.d;
                 ep.n_b = 1; ep.b_rows[0] = md.d;
                 CUtensorMap tb[3] = {c->tm_w[W_WO][l], c->tm_w[W_WO][l], c->tm_w[W_WO][l]};
-                { Timed tm(c, 5, s); st = launch_gemm_tc(c->tm_a_q, tb, ep, c->d_status, c->n_sms, s, &c->tm_h, c->gemm_impl == 2); }
+                { Timed tm(c, 5, s); st = launch_gemm_tc(c->tm_a_q, tb, ep, c->d_status, c->n_sms, s, tp ? nullptr : &c->tm_h, c->gemm_impl == 2); }
                 if (st != KVR_OK) return st;
             } else {
                 Timed tm(c, 5, s);
-                launch_gemm_simt(fp32, 1, a, md.q_dim, c->w[W_WO][l], nullptr, md.q_dim, n, md.d, md.q_dim, h, md.d,
-                                 s);
+                launch_gemm_simt(fp32, tp ? 0 : 1, a, md.q_dim, c->w[W_WO][l], nullptr, md.q_dim, n, md.d, md.q_dim,
+                                 tp ? part : h, md.d, s);
             }
             ++launches;
-            { Timed tm(c, 2, s); launch_rmsnorm(fp32, h, c->w[W_LN2][l], a, n, md.d, md.eps, s); } ++launches;
+            if (tp) {
+                if ((st = tp_allreduce()) != KVR_OK) return st;
+                Timed tm(c, 2, s);
+                launch_add_rmsnorm(fp32, h, part, c->w[W_LN2][l], a, n, md.d, md.eps, s);
+            } else {
+                Timed tm(c, 2, s);
+                launch_rmsnorm(fp32, h, c->w[W_LN2][l], a, n, md.d, md.eps, s);
+            }
+            ++launches;
             // gate/up + SwiGLU, then down + residual
             if (use_tc_gemm) {
                 TcGemmEpilogue ep{};
@@ -798,18 +862,24 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
                 { Timed tm(c, 6, s); st = launch_gemm_tc(c->tm_a_d, tb, ep, c->d_status, c->n_sms, s, nullptr, c->gemm_impl == 2); }
                 if (st != KVR_OK) return st;
                 TcGemmEpilogue e2{};
-                e2.mode = TC_RESID; e2.M = n; e2.N = md.d; e2.K = md.F; e2.c_f32 = h; e2.ldc = md.d;
+                e2.mode = tp ? TC_STORE_F32 : TC_RESID; e2.M = n; e2.N = md.d; e2.K = md.F;
+                e2.c_f32 = tp ? part : h; e2.ldc = md.d;
                 e2.n_b = 1; e2.b_rows[0] = md.d;
                 CUtensorMap tb2[3] = {c->tm_w[W_WD][l], c->tm_w[W_WD][l], c->tm_w[W_WD][l]};
-                { Timed tm(c, 7, s); st = launch_gemm_tc(c->tm_m, tb2, e2, c->d_status, c->n_sms, s, &c->tm_h, c->gemm_impl == 2); }
+                { Timed tm(c, 7, s); st = launch_gemm_tc(c->tm_m, tb2, e2, c->d_status, c->n_sms, s, tp ? nullptr : &c->tm_h, c->gemm_impl == 2); }
                 if (st != KVR_OK) return st;
             } else {
                 { Timed tm(c, 6, s);
                   launch_gemm_simt(fp32, 2, a, md.d, c->w[W_WG][l], c->w[W_WU][l], md.d, n, md.F, md.d, m, md.F, s); }
                 { Timed tm(c, 7, s);
-                  launch_gemm_simt(fp32, 1, m, md.F, c->w[W_WD][l], nullptr, md.F, n, md.d, md.F, h, md.d, s); }
+                  launch_gemm_simt(fp32, tp ? 0 : 1, m, md.F, c->w[W_WD][l], nullptr, md.F, n, md.d, md.F,
+                                   tp ? part : h, md.d, s); }
             }
             launches += 2;
+            if (tp) {   // summed over the ranks now, added to the residual by the next layer's norm
+                if ((st = tp_allreduce()) != KVR_OK) return st;
+                tp_pending = true;
+            }
         }
     }
     CU_OK(cudaEventRecord(c->staging_free, s));
@@ -892,6 +962,7 @@ int kv_sync_status(kvr_ctx *c, void *stream) {
 int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, float *logits_out, void *stream) {
     if (!c || !final_gain || !lm_head || !logits_out) return KVR_ERR_INVALID_ARG;
     if (!c->arena_bound || !c->weights_bound || !c->ws_bound) return KVR_ERR_NOT_BOUND;
+    if (c->tp_world > 1) return KVR_ERR_UNSUPPORTED;   // the last layer's reductions and a sharded head are not built
     if (!c->have_last) return KVR_ERR_NOT_BOUND;   // no rebuild with "keep_last_hidden" came before
     const ModelDims &md = c->md;
     const bool fp32 = is_fp32(c);

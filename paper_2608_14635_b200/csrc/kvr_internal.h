@@ -54,6 +54,10 @@ void launch_embed_rmsnorm(bool fp32, const void *embed, const void *gain, const 
                           void *a, int d, float eps, cudaStream_t s);
 void launch_rmsnorm(bool fp32, const float *h, const void *gain, void *a, int n, int d, float eps,
                     cudaStream_t s);
+// h += part (both fp32 [n, d]), then a = rmsnorm(h) * gain: the residual add of a tensor-parallel partial sum
+// folded into the norm that follows it
+void launch_add_rmsnorm(bool fp32, float *h, const float *part, const void *gain, void *a, int n, int d, float eps,
+                        cudaStream_t s);
 void launch_rope_table(const int32_t *pos, int n, int hd, const RopeFreq &f, float2 *cs, cudaStream_t s);
 // mode 0: C fp32 [M, ldc] = A W0^T; 1: C fp32 += A W0^T; 2: C (T) = silu(A W0^T) * (A W1^T)
 void launch_gemm_simt(bool fp32, int mode, const void *A, int lda, const void *W0, const void *W1, int ldw,

@@ -148,6 +148,47 @@ __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restric
     }
 }
 
+// h += part, then the norm of the updated row (tensor-parallel ranks: `part` is the all-reduced
+// partial product of the preceding row-parallel projection).
+template <typename T>
+__global__ void __launch_bounds__(256) add_rmsnorm_kernel(float *__restrict__ h, const float *__restrict__ part,
+                                                          const T *__restrict__ gain, T *__restrict__ a, int d,
+                                                          float eps) {
+    constexpr int VEC = sizeof(T) == 4 ? 4 : 8;
+    extern __shared__ float row[];
+    __shared__ float red[32];
+    const int64_t t = blockIdx.x;
+    float ss = 0.f;
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+        float4 x = *reinterpret_cast<const float4 *>(h + t * d + i);
+        const float4 y = *reinterpret_cast<const float4 *>(part + t * d + i);
+        x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+        *reinterpret_cast<float4 *>(h + t * d + i) = x;
+        *reinterpret_cast<float4 *>(row + i) = x;
+        ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+    }
+    ss = block_sum(ss, red);
+    const float rstd = 1.0f / sqrtf(ss / (float)d + eps);
+    for (int i = threadIdx.x * VEC; i < d; i += blockDim.x * VEC) {
+        float g[VEC], o[VEC];
+        load_vec<T, VEC>(gain + i, g);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) o[j] = row[i + j] * rstd * g[j];
+        store_vec<T, VEC>(a + t * d + i, o);
+    }
+}
+
+void launch_add_rmsnorm(bool fp32, float *h, const float *part, const void *gain, void *a, int n, int d, float eps,
+                        cudaStream_t s) {
+    if (n == 0) return;
+    const size_t sm = (size_t)d * sizeof(float);
+    if (fp32)
+        add_rmsnorm_kernel<float><<<n, 256, sm, s>>>(h, part, (const float *)gain, (float *)a, d, eps);
+    else
+        add_rmsnorm_kernel<__nv_bfloat16><<<n, 256, sm, s>>>(h, part, (const __nv_bfloat16 *)gain,
+                                                              (__nv_bfloat16 *)a, d, eps);
+}
+
 void launch_embed_rmsnorm(bool fp32, const void *embed, const void *gain, const ChunkMeta &cm, float *h,
                           void *a, int d, float eps, cudaStream_t s) {
     if (cm.n == 0) return;
