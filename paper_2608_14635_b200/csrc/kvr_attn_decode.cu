@@ -74,7 +74,7 @@ attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *_
         if (live) {
             slot = (int64_t)tab[key / block_size] * block_size + (key % block_size);
             const uint4 *kr = reinterpret_cast<const uint4 *>(arena_k + slot * kv_dim + hk * HD);
-#pragma unroll 4
+#pragma unroll 8
             for (int c = 0; c < HD / 8; ++c) {
                 float kf[8];
                 bf16x8_to_f32(kr[c], kf);
@@ -112,9 +112,12 @@ attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *_
 #pragma unroll
                 for (int e = 0; e < EPL; ++e) acc[g][e] *= corr[g];
             }
+        // All 32 keys of the block, eight value rows in flight at a time: a key past the end has
+        // probability 0 and borrows the address of the block's last live key (its own slot may hold anything).
         const int n_live = min(32, k1 - kb);
-        for (int kk = 0; kk < n_live; ++kk) {
-            const int64_t sl = __shfl_sync(0xffffffffu, slot, kk);
+#pragma unroll 8
+        for (int kk = 0; kk < 32; ++kk) {
+            const int64_t sl = __shfl_sync(0xffffffffu, slot, min(kk, n_live - 1));
             const __nv_bfloat16 *vr = arena_k + kv_stride + sl * kv_dim + hk * HD + lane * EPL;
             float vf[EPL];
             if (EPL == 4) {
