@@ -53,7 +53,9 @@ __device__ __forceinline__ bool loads_muted(const int *status) {
 // first probe has failed).  Returns false (and records the failure in *status)
 // if the limit expires, so that no wait can hang the GPU.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int *status, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+    // fast path: a few dozen probes with nothing else in the loop (no clock reads, no global loads)
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
     const long long limit = *reinterpret_cast<const volatile long long *>(status + STATUS_LIMIT);
     const long long t0 = clock64();
     while (true) {
