@@ -291,8 +291,8 @@ attn_fa_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             ptx::mbar_init(b_kfree + 8 * s, 1);
             ptx::mbar_init(b_vfree + 8 * s, 1);
             ptx::mbar_init(b_sfull + 8 * s, 1);
-            ptx::mbar_init(b_pready + 8 * s, FA_SM_WARPS / 2);   // P of keys 0..63: one arrival per softmax warp
-            ptx::mbar_init(b_phi + 8 * s, FA_SM_WARPS / 2);      // P of keys 64..127
+            ptx::mbar_init(b_pready + 8 * s, FA_SM_WARPS / 2 * 32);   // P of keys 0..63: one arrival per softmax thread
+            ptx::mbar_init(b_phi + 8 * s, FA_SM_WARPS / 2 * 32);      // P of keys 64..127
             ptx::mbar_init(b_ofull + 8 * s, 1);
         }
         ptx::mbar_init(b_vzero, 1);
@@ -502,14 +502,12 @@ attn_fa_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             tmem_st16(tSx + 16 * half, pk);
             ptx::tmem_st_wait();
             ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(b_pready + 8 * x);
+            ptx::mbar_arrive(b_pready + 8 * x);
             l_sum += exp_chunk(r[1], scale_log2, msc, pk);
             tmem_st16(tSx + 16 * half + 32, pk);
             ptx::tmem_st_wait();
             ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(b_phi + 8 * x);
+            ptx::mbar_arrive(b_phi + 8 * x);
         }
         // row sum = both halves' (slots of their own: the partner may still be reading the last max)
         my_x[4 * FA_M] = l_sum;
