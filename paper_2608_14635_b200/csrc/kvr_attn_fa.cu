@@ -339,20 +339,20 @@ attn_fa_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (lane == 0) ptx::mbar_expect_tx(b_kfull + 8 * s, nblk * HALVES * FA_BLOCK * 128);
             __syncwarp();
             if (mine)
-                ptx::tma_load_4d(sK[s] + dst_off, &tmKV, 0, 0, hk * HALVES, (p.k_row0 + blk * FA_BLOCK) >> 3,
+                ptx::tma_load_4d((s ? sK[1] : sK[0]) + dst_off, &tmKV, 0, 0, hk * HALVES, (p.k_row0 + blk * FA_BLOCK) >> 3,
                                  b_kfull + 8 * s);
             if (!ptx::mbar_wait(b_vfree + 8 * s, ph ^ 1u, p.status, abort_flag)) { ok = false; break; }
             if (lane == 0) ptx::mbar_expect_tx(b_vfull + 8 * s, nblk * HALVES * FA_BLOCK * 128);
             __syncwarp();
             if (mine)
-                ptx::tma_load_4d(sV[s] + dst_off, &tmKV, 0, 0, hk * HALVES, (p.v_row0 + blk * FA_BLOCK) >> 3,
+                ptx::tma_load_4d((s ? sV[1] : sV[0]) + dst_off, &tmKV, 0, 0, hk * HALVES, (p.v_row0 + blk * FA_BLOCK) >> 3,
                                  b_vfull + 8 * s);
             if (tail && j == n_steps - 1) {
                 // V rows past the prefix may hold anything (NaN included): zero them so
                 // that their zero probabilities cannot poison the PV product.
                 if (!ptx::mbar_wait(b_vfull + 8 * s, ph, p.status, abort_flag)) { ok = false; break; }
                 const int r0 = kv_len - j * FA_N;
-                uint8_t *vst = smem_raw + (sV[s] - ptx::smem_u32(smem_raw));
+                uint8_t *vst = smem_raw + ((s ? sV[1] : sV[0]) - ptx::smem_u32(smem_raw));
                 const int n16 = (FA_N - r0) * HALVES * 8;
                 for (int i = lane; i < n16; i += 32) {
                     const int r = r0 + i / (HALVES * 8), h = (i / 8) % HALVES, q = i % 8;
@@ -374,15 +374,16 @@ attn_fa_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint32_t tS[2] = {tmem, tmem + 256}, tO[2] = {tmem + 128, tmem + 384};
             const int n_x[2] = {n_a, n_b};
             bool ok = ptx::mbar_wait(b_qfull, 0, p.status, abort_flag);
-            // descriptors are built once; per MMA only the 16-byte address field moves
-            const uint64_t qd[2] = {ptx::smem_desc_sw128(sQ[0]), ptx::smem_desc_sw128(sQ[1])};
-            const uint64_t kd[2] = {smem_desc_k_sw128(sK[0], GROUP), smem_desc_k_sw128(sK[1], GROUP)};
-            const uint64_t vd[2] = {smem_desc_mn_sw128(sV[0], GROUP), smem_desc_mn_sw128(sV[1], GROUP)};
+            // descriptors are built once; per MMA only the 16-byte address field moves (scalars chosen by a
+            // select, not arrays indexed by the stage: an indexed array would live in local memory)
+            const uint64_t qd0 = ptx::smem_desc_sw128(sQ[0]), qd1 = ptx::smem_desc_sw128(sQ[1]);
+            const uint64_t kd0 = smem_desc_k_sw128(sK[0], GROUP), kd1 = smem_desc_k_sw128(sK[1], GROUP);
+            const uint64_t vd0 = smem_desc_mn_sw128(sV[0], GROUP), vd1 = smem_desc_mn_sw128(sV[1], GROUP);
             auto issue_qk = [&](int x, int j) {
-                const int s = j & 1;
+                const uint64_t kd = (j & 1) ? kd1 : kd0, qd = x ? qd1 : qd0;
                 {
-                    if (HD == 128) mma_group_qk128(tS[x], qd[x], kd[s], IDESC_QK, 0);
-                    else mma_group_qk64(tS[x], qd[x], kd[s], IDESC_QK, 0);
+                    if (HD == 128) mma_group_qk128(x ? tmem + 256 : tmem, qd, kd, IDESC_QK, 0);
+                    else mma_group_qk64(x ? tmem + 256 : tmem, qd, kd, IDESC_QK, 0);
                     ptx::mma_commit(b_sfull + 8 * x);
                 }
             };
@@ -396,6 +397,7 @@ attn_fa_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             for (int j = 0; j < n_steps && ok; ++j) {
                 const int s = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+                const uint64_t vd = s ? vd1 : vd0;
                 // The loads of this step's V and the next step's K landed long ago: their barriers are
                 // polled first, while the previous step's last MMAs still run, so that between the
                 // groups below only the wait for P stands.
@@ -418,16 +420,15 @@ attn_fa_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (!(x == x_first && p_in) &&
                         !ptx::mbar_wait(b_pready + 8 * x, (uint32_t)j & 1u, p.status, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after();
-                    if (HD == 128) mma_group_pv128_half(tO[x], tS[x], vd[s], IDESC_PV, j != 0);
-                    else mma_group_pv64_half(tO[x], tS[x], vd[s], IDESC_PV, j != 0);
+                    if (HD == 128) mma_group_pv128_half(tO[x], tS[x], vd, IDESC_PV, j != 0);
+                    else mma_group_pv64_half(tO[x], tS[x], vd, IDESC_PV, j != 0);
                     if (!ptx::mbar_wait(b_phi + 8 * x, (uint32_t)j & 1u, p.status, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after();
-                    if (HD == 128) mma_group_pv128_half(tO[x], tS[x] + 32, vd[s] + 1024, IDESC_PV, 1);
-                    else mma_group_pv64_half(tO[x], tS[x] + 32, vd[s] + 512, IDESC_PV, 1);
+                    if (HD == 128) mma_group_pv128_half(tO[x], tS[x] + 32, vd + 1024, IDESC_PV, 1);
+                    else mma_group_pv64_half(tO[x], tS[x] + 32, vd + 512, IDESC_PV, 1);
                     if (j == n_x[x] - 1) ptx::mma_commit(b_ofull + 8 * x);
                     // next step's scores for this sub-tile
                     if (j + 1 < n_x[x]) {
-                        const int s1 = (j + 1) & 1;
                         issue_qk(x, j + 1);
                     }
                 }
