@@ -82,6 +82,7 @@ struct kvr_ctx {
     // resume logits: residual rows of every request's final token, kept by the last rebuild
     int keep_last = 0;
     bool have_last = false;
+    bool dev_tables_current = false;   // the workspace still holds the last rebuild's block tables
     std::vector<int32_t> last_lens, last_tables;
     int32_t last_width = 0;
     CUtensorMap tm_la_d{}, tm_la_q{}, tm_lm{}, tm_lq{}, tm_lh{};
@@ -568,6 +569,7 @@ int kv_workspace_bind(kvr_ctx *c, void *ws, size_t bytes, int64_t max_chunk_toke
         if (st != KVR_OK) return st;
     }
     c->ws_bound = true;
+    c->dev_tables_current = false;
     return KVR_OK;
 }
 
@@ -648,6 +650,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     for (int r = 0; r < R; ++r) T += lens[r] - skip[r];
     c->last_computed = T;
     c->have_last = false;
+    c->dev_tables_current = false;
     c->last_chunks = 0;
     c->last_launches = 0;
     c->ev_kind.clear();
@@ -886,6 +889,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     c->staging_busy = true;
     c->last_chunks = n_chunks;
     c->last_launches = launches;
+    c->dev_tables_current = true;
     if (c->keep_last) {
         bool all = true;
         for (int r = 0; r < R; ++r) all = all && lens[r] > 0;
@@ -920,6 +924,7 @@ static int readback_common(kvr_ctx *c, int32_t layer, const int32_t *table, int3
     if (st != KVR_OK) return st;
     std::memcpy(c->pinned, table, (size_t)need * sizeof(int32_t));
     int32_t *d_tab = (int32_t *)(c->ws + c->lay.tables);
+    c->dev_tables_current = false;   // this call's table goes over them
     CU_OK(cudaMemcpyAsync(d_tab, c->pinned, (size_t)need * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     CU_OK(cudaEventRecord(c->staging_free, s));
     c->staging_busy = true;
@@ -991,14 +996,17 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     int32_t *st_tab = (int32_t *)c->pinned;
     int32_t *st_pos = (int32_t *)(c->pinned + align_up(tb));
     AttnTile *st_tiles = (AttnTile *)(c->pinned + align_up(tb) + align_up((size_t)R * 2 * sizeof(int32_t)));
-    std::memcpy(st_tab, c->last_tables.data(), tb);
+    // the block tables are still in the workspace when nothing but the rebuild has used it since
+    const bool copy_tables = !c->dev_tables_current;
+    if (copy_tables) std::memcpy(st_tab, c->last_tables.data(), tb);
     for (int r = 0; r < R; ++r) {
         st_pos[r] = c->last_lens[r] - 1;
         st_pos[R + r] = r;
         st_tiles[r] = AttnTile{r, c->last_lens[r] - 1, 1, r};
     }
     std::stable_sort(st_tiles, st_tiles + R, [](const AttnTile &x, const AttnTile &y) { return x.pos0 > y.pos0; });
-    CU_OK(cudaMemcpyAsync(d_tables, st_tab, tb, cudaMemcpyHostToDevice, s));
+    if (copy_tables) CU_OK(cudaMemcpyAsync(d_tables, st_tab, tb, cudaMemcpyHostToDevice, s));
+    c->dev_tables_current = true;
     CU_OK(cudaMemcpyAsync(d_pos, st_pos, (size_t)R * 2 * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     CU_OK(cudaMemcpyAsync(d_tiles, st_tiles, (size_t)R * sizeof(AttnTile), cudaMemcpyHostToDevice, s));
     CU_OK(cudaEventRecord(c->staging_free, s));
