@@ -251,7 +251,8 @@ int kv_readback_noalloc(const void *arena_dev, const kv_arena_geometry *geom, in
  * `lm_head_dev` [vocab, d_model] (both in the model's dtype, 16-byte aligned):
  *     logits_out_dev[r, :] (fp32, [R, vocab])   for the R requests of that rebuild, in order.
  * Every request of the rebuild must have had a non-empty prefix.  Enqueues on `stream`;
- * KVR_ERR_NOT_BOUND if no such rebuild came before. */
+ * KVR_ERR_NOT_BOUND if no such rebuild came before.  The kept rows are only read: the call
+ * can be repeated after one rebuild and gives the same logits each time. */
 int kv_resume_logits(kvr_ctx *ctx, const void *final_gain_dev, const void *lm_head_dev, float *logits_out_dev,
                      void *stream);
 
@@ -322,7 +323,9 @@ int kv_debug_profile(kvr_ctx *ctx, double *ms_by_kind, int64_t *launches_by_kind
  * written; default 0); "profile" 0/1 (see kv_debug_profile; default 0); "gemm" 0 = plain-FMA kernels,
  * 1 = tcgen05 kernels on 128 x 256 tiles, 2 = tcgen05 kernels on CTA pairs (256 x 256 tiles); 1 and 2 are bf16 only, 2 is the default in bf16;
  * "attn" 0 = plain kernel, 1 = warp-level MMA kernel, 2 = tcgen05 kernel (1 and 2 bf16 only; 2 is the
- * default in bf16 and needs block_size 16, otherwise 1 is used).
+ * default in bf16 and needs block_size 16, otherwise 1 is used); "resume_gemm" 0/1 (kv_resume_logits with the tcgen05
+ * kernels and at most 128 requests: 1 = projections by the weight-streaming kernel that cuts the grid along the weight rows
+ * and K, the default; 0 = by the rebuild's GEMM).
  * Returns KVR_ERR_INVALID_ARG for unknown names or values. */
 int kv_set_option(kvr_ctx *ctx, const char *name, int64_t value);
 

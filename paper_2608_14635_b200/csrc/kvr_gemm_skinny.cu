@@ -1,0 +1,201 @@
+// Weight-streaming GEMM for a handful of activation rows (the R final-token rows of
+// kv_resume_logits, R <= 128):  out[r, n] = sum_k X[r, k] W[n, k].
+// With so few rows the product is bound by reading W once from HBM, so the grid is cut
+// along the weight rows (and, for matrices with few rows, along K) instead of along R:
+//   - the operands are swapped on the tensor core: the 128 weight rows of a CTA's tile are
+//     the MMA's M, the requests are its N (padded to a multiple of 16), so the accumulator
+//     in TMEM is out^T: lane = weight row n, column = request r, and a warp's store of one
+//     column writes 32 consecutive n of one output row;
+//   - one tile per CTA, grid (ceil(N / 128), splits); a split covers a contiguous range of
+//     64-wide K blocks and writes its fp32 partial product to out + split * split_stride,
+//     which the consumer kernel sums in a fixed order (no atomics, run-to-run identical);
+//   - a TMA ring of six 32 KB stages (four 48 KB stages for the SwiGLU pair) keeps about
+//     100 KB of weight bytes in flight per SM.
+// Warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue.
+// Every wait is bounded through the context's status block, as in the large GEMM.
+#include "kvr_internal.h"
+#include "kvr_ptx.cuh"
+
+namespace kvr {
+
+namespace {
+
+constexpr int SK_ROWS = 128, SK_BK = 64, SK_UMMA_K = 16;
+constexpr int SK_TILE_BYTES = SK_ROWS * SK_BK * 2;   // one 128 x 64 bf16 box
+constexpr int SK_THREADS = 192;
+
+template <bool SWIGLU>
+struct SkCfg {
+    static constexpr int STAGES = SWIGLU ? 4 : 6;
+    static constexpr int N_W = SWIGLU ? 2 : 1;                       // weight boxes per stage
+    static constexpr int STAGE_BYTES = (N_W + 1) * SK_TILE_BYTES;    // weights, then the activation box
+    static constexpr int TMEM_COLS = SWIGLU ? 256 : 128;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+};
+
+template <bool SWIGLU>
+__global__ void __launch_bounds__(SK_THREADS, 1)
+gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
+                   const __grid_constant__ CUtensorMap tmW1, const SkinnyArgs a, int *status) {
+    using Cfg = SkCfg<SWIGLU>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = ptx::smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    const uint32_t bars = tiles + Cfg::STAGES * Cfg::STAGE_BYTES;
+    const uint32_t full0 = bars, empty0 = bars + 8 * Cfg::STAGES, tfull = bars + 16 * Cfg::STAGES;
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ int abort_sh;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_sh = 0;
+        for (int s = 0; s < Cfg::STAGES; ++s) {
+            ptx::mbar_init(full0 + 8 * s, 1);
+            ptx::mbar_init(empty0 + 8 * s, 1);
+        }
+        ptx::mbar_init(tfull, 1);
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmX);
+        ptx::prefetch_tmap(&tmW0);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&tmem_base_sh), Cfg::TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sh;
+    volatile int *abort_flag = &abort_sh;
+
+    const int tile = blockIdx.x, split = blockIdx.y, n_split = gridDim.y;
+    const int num_k = (a.K + SK_BK - 1) / SK_BK;
+    const int kb0 = (int)((int64_t)split * num_k / n_split), kb1 = (int)((int64_t)(split + 1) * num_k / n_split);
+    const bool empty = kb1 <= kb0;   // more splits than K blocks: this split's partial product is zero
+    const int n_pad = a.R <= 16 ? 16 : ((a.R + 15) & ~15);
+
+    if (warp == 0) {
+        if (lane == 0 && !empty && !ptx::loads_muted(status)) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1u, status, abort_flag)) break;
+                const uint32_t fb = full0 + 8 * stage;
+                const uint32_t sa = tiles + stage * Cfg::STAGE_BYTES;
+                ptx::mbar_expect_tx(fb, Cfg::STAGE_BYTES);
+                ptx::tma_load_2d(sa, &tmW0, kb * SK_BK, tile * SK_ROWS, fb);
+                if (SWIGLU) ptx::tma_load_2d(sa + SK_TILE_BYTES, &tmW1, kb * SK_BK, tile * SK_ROWS, fb);
+                ptx::tma_load_2d(sa + Cfg::N_W * SK_TILE_BYTES, &tmX, kb * SK_BK, 0, fb);
+                if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && !empty) {
+            const uint32_t idesc = ptx::idesc_bf16(SK_ROWS, n_pad);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!ptx::mbar_wait(full0 + 8 * stage, phase, status, abort_flag)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t sa = tiles + stage * Cfg::STAGE_BYTES;
+                const uint64_t dw0 = ptx::smem_desc_sw128(sa);
+                const uint64_t dw1 = ptx::smem_desc_sw128(sa + SK_TILE_BYTES);
+                const uint64_t dx = ptx::smem_desc_sw128(sa + Cfg::N_W * SK_TILE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < SK_BK / SK_UMMA_K; ++kk) {
+                    const uint32_t accum = (kb > kb0 || kk > 0) ? 1u : 0u;
+                    ptx::mma_bf16_ss(tmem_base, dw0 + 2 * kk, dx + 2 * kk, idesc, accum);
+                    if (SWIGLU) ptx::mma_bf16_ss(tmem_base + 128, dw1 + 2 * kk, dx + 2 * kk, idesc, accum);
+                }
+                ptx::mma_commit(empty0 + 8 * stage);
+                if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) ptx::mma_commit(tfull);
+        }
+    } else {
+        const int quarter = warp & 3;   // the 32 TMEM lanes this warp may read
+        const int n = tile * SK_ROWS + quarter * 32 + lane;
+        bool ok = true;
+        if (!empty) {
+            ok = ptx::mbar_wait(tfull, 0, status, abort_flag);
+            ptx::tc_fence_after();
+        }
+        if (ok) {
+            const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < n_pad; c += 16) {
+                uint32_t g[16], u[16];
+                if (!empty) {
+                    ptx::tmem_ld16(tacc + c, g);
+                    if (SWIGLU) ptx::tmem_ld16(tacc + 128 + c, u);
+                    ptx::tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) g[j] = u[j] = 0u;
+                }
+                if (n >= a.N) {
+                    // rows of the last tile past the matrix: nothing to store
+                } else if (SWIGLU) {
+                    __nv_bfloat16 *dst = a.out_bf16 + n;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        if (c + j < a.R) {
+                            const float gv = __uint_as_float(g[j]);
+                            const float sv = gv / (1.0f + __expf(-gv));
+                            dst[(int64_t)(c + j) * a.ld_bf16] = __float2bfloat16_rn(sv * __uint_as_float(u[j]));
+                        }
+                    }
+                } else {
+                    float *dst = a.out_f32 + (int64_t)split * a.split_stride + n;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c + j < a.R) dst[(int64_t)(c + j) * a.ldo] = __uint_as_float(g[j]);
+                }
+                __syncwarp();
+            }
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+int gemm_skinny_init(int device) {
+    (void)device;
+    if (cudaFuncSetAttribute(gemm_skinny_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SkCfg<false>::SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_skinny_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SkCfg<true>::SMEM_BYTES) != cudaSuccess)
+        return KVR_ERR_CUDA;
+    return KVR_OK;
+}
+
+// One wave of CTAs where the matrix has fewer 128-row tiles than the GPU has SMs.
+int gemm_skinny_splits(int N, int K, int n_sms) {
+    const int tiles = (N + SK_ROWS - 1) / SK_ROWS, num_k = (K + SK_BK - 1) / SK_BK;
+    int s = n_sms / (tiles > 0 ? tiles : 1);
+    if (s > GEMM_SKINNY_MAX_SPLITS) s = GEMM_SKINNY_MAX_SPLITS;
+    if (s > num_k) s = num_k;
+    return s < 1 ? 1 : s;
+}
+
+int launch_gemm_skinny(const CUtensorMap &tmX, const CUtensorMap &tmW0, const CUtensorMap *tmW1,
+                       const SkinnyArgs &a, int splits, int *d_status, cudaStream_t s) {
+    if (a.R <= 0 || a.N <= 0) return KVR_OK;
+    if (a.R > GEMM_SKINNY_MAX_ROWS || a.K <= 0 || splits < 1 || splits > GEMM_SKINNY_MAX_SPLITS)
+        return KVR_ERR_UNSUPPORTED;
+    const dim3 grid((a.N + SK_ROWS - 1) / SK_ROWS, tmW1 ? 1 : splits);
+    if (tmW1)
+        gemm_skinny_kernel<true><<<grid, SK_THREADS, SkCfg<true>::SMEM_BYTES, s>>>(tmX, tmW0, *tmW1, a, d_status);
+    else
+        gemm_skinny_kernel<false><<<grid, SK_THREADS, SkCfg<false>::SMEM_BYTES, s>>>(tmX, tmW0, tmW0, a, d_status);
+    return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
+}
+
+}  // namespace kvr

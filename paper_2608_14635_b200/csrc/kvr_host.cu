@@ -19,7 +19,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct WsLayout {
     size_t h, a, q, m, cs, meta, tables, tiles, part, total;
-    size_t l_h, l_a, l_q, l_m, l_cs, l_pos, l_pairs, l_tiles, l_part;   // per-request buffers for kv_resume_logits
+    size_t l_h, l_h2, l_sk, l_a, l_q, l_m, l_cs, l_pos, l_pairs, l_tiles, l_part;   // per-request buffers for kv_resume_logits
     size_t m_bytes;
 };
 
@@ -70,6 +70,7 @@ struct kvr_ctx {
     void *tp_user = nullptr;
     // options
     int gemm_impl = 2, attn_impl = 2, profile = 0, probe_mute = 0;
+    int resume_gemm = 1;           // kv_resume_logits: 1 = weight-streaming GEMM for up to 128 requests, 0 = the rebuild's GEMM
     uint32_t *d_probe = nullptr;   // [2 * PROBE_MAX_BLOCKS]: flags, results
     uint32_t probe_epoch = 0;      // word the current probe publishes; never 0, never reused by the next call
     int clock_khz = 0;
@@ -140,7 +141,10 @@ bool compute_layout(const kvr_ctx *c, int64_t Tc, int32_t max_req, int32_t max_b
     const size_t max_tiles = T / ATTN_TILE_Q + (size_t)max_req + 1;
     L->tiles = o; o += align_up(max_tiles * sizeof(AttnTile));
     const size_t Rq = (size_t)max_req;
-    L->l_h = o; o += align_up(Rq * md.d * sizeof(float));
+    L->l_h = o; o += align_up(Rq * md.d * sizeof(float));    // kept by the rebuild, read-only for the resume call
+    L->l_h2 = o; o += align_up(Rq * md.d * sizeof(float));   // the resume call's own residual rows
+    L->l_sk = o;   // partial products of the K splits of the weight-streaming GEMM
+    o += align_up((size_t)GEMM_SKINNY_MAX_SPLITS * Rq * (size_t)std::max(md.d, md.q_dim) * sizeof(float));
     L->l_a = o; o += align_up(Rq * (size_t)std::max(md.d, md.q_dim) * es);
     L->l_q = o; o += align_up(Rq * (size_t)md.q_dim * es);
     L->l_m = o; o += align_up(std::max(Rq * (size_t)md.F * es, Rq * (size_t)md.q_dim * sizeof(float)));
@@ -367,7 +371,7 @@ int kv_ctx_create(kvr_ctx **out, int device) {
         return KVR_ERR_CUDA;
     }
     c->tc_ready = (prop.major == 10) && tc_gemm_init(device) == KVR_OK && attn_tc_init(device) == KVR_OK &&
-                  attn_fa_init(device) == KVR_OK;
+                  attn_fa_init(device) == KVR_OK && gemm_skinny_init(device) == KVR_OK;
     *out = c;
     return KVR_OK;
 }
@@ -565,7 +569,7 @@ int kv_workspace_bind(kvr_ctx *c, void *ws, size_t bytes, int64_t max_chunk_toke
         if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_la_q, c->ws + L.l_a, max_requests, md.q_dim, 128, 64);
         if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_lm, c->ws + L.l_m, max_requests, md.F, 128, 64);
         if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_lq, c->ws + L.l_q, max_requests, md.q_dim, 128, 64);
-        if (st == KVR_OK) st = tc_make_tmap_f32(&c->tm_lh, c->ws + L.l_h, max_requests, md.d);
+        if (st == KVR_OK) st = tc_make_tmap_f32(&c->tm_lh, c->ws + L.l_h2, max_requests, md.d);
         if (st != KVR_OK) return st;
     }
     c->ws_bound = true;
@@ -583,6 +587,11 @@ int kv_set_option(kvr_ctx *c, const char *name, int64_t value) {
     if (!std::strcmp(name, "gemm")) {
         if (value < 0 || value > 2) return KVR_ERR_INVALID_ARG;
         c->gemm_impl = (int)value;
+        return KVR_OK;
+    }
+    if (!std::strcmp(name, "resume_gemm")) {
+        if (value < 0 || value > 1) return KVR_ERR_INVALID_ARG;
+        c->resume_gemm = (int)value;
         return KVR_OK;
     }
     if (!std::strcmp(name, "wait_limit_ms")) {
@@ -766,7 +775,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
             {
                 Timed tm(c, l == 0 ? 1 : 2, s);
                 if (l == 0) launch_embed_rmsnorm(fp32, c->embed, c->w[W_LN1][0], cm, h, a, md.d, md.eps, s);
-                else if (tp_pending) launch_add_rmsnorm(fp32, h, part, c->w[W_LN1][l], a, n, md.d, md.eps, s);
+                else if (tp_pending) launch_add_rmsnorm(fp32, h, h, part, 1, 0, c->w[W_LN1][l], a, n, md.d, md.eps, s);
                 else launch_rmsnorm(fp32, h, c->w[W_LN1][l], a, n, md.d, md.eps, s);
                 tp_pending = false;
             }
@@ -849,7 +858,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
             if (tp) {
                 if ((st = tp_allreduce()) != KVR_OK) return st;
                 Timed tm(c, 2, s);
-                launch_add_rmsnorm(fp32, h, part, c->w[W_LN2][l], a, n, md.d, md.eps, s);
+                launch_add_rmsnorm(fp32, h, h, part, 1, 0, c->w[W_LN2][l], a, n, md.d, md.eps, s);
             } else {
                 Timed tm(c, 2, s);
                 launch_rmsnorm(fp32, h, c->w[W_LN2][l], a, n, md.d, md.eps, s);
@@ -982,7 +991,10 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     const int R = (int)c->last_lens.size(), width = c->last_width, l = md.L - 1;
     char *ws = c->ws;
     const WsLayout &L = c->lay;
-    float *h = (float *)(ws + L.l_h);
+    // the rows the rebuild kept stay as they are (the call can be repeated); h is this call's residual
+    const float *h0 = (const float *)(ws + L.l_h);
+    float *h = (float *)(ws + L.l_h2);
+    float *sk = (float *)(ws + L.l_sk);
     void *a = ws + L.l_a, *q = ws + L.l_q, *m = ws + L.l_m;
     float2 *cs = (float2 *)(ws + L.l_cs);
     int32_t *d_pos = (int32_t *)(ws + L.l_pos), *d_row = d_pos + R;
@@ -1015,11 +1027,25 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     for (int i = 0; i < md.hd / 2; ++i) rf.inv_freq[i] = std::pow(md.rope_base, -2.0 * i / md.hd);
     ChunkMeta cm{d_pos, d_pos, d_pos, d_row, R};   // tok and slot are not used on this path
     launch_rope_table(d_pos, R, md.hd, rf, cs, s);
-    launch_rmsnorm(fp32, h, c->w[W_LN1][l], a, R, md.d, md.eps, s);
+    // few rows: every projection is bound by reading its weights once, which the weight-streaming GEMM does
+    // on all SMs; its K splits leave fp32 partial products that the next kernel sums
+    const bool use_sk = use_tc && c->resume_gemm == 1 && R <= GEMM_SKINNY_MAX_ROWS;
+    if (!use_sk) CU_OK(cudaMemcpyAsync(h, h0, (size_t)R * md.d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    launch_rmsnorm(fp32, h0, c->w[W_LN1][l], a, R, md.d, md.eps, s);
     // q of the final tokens (RoPE at position len - 1); their K/V are already in the arena
     QkvExtras ex = qkv_extras(c, l);
     ex.bk = ex.bv = ex.kn = nullptr;   // only q is projected here
-    if (use_tc_q) {
+    ModelDims q_only = md;
+    q_only.Hkv = 0; q_only.kv_dim = 0;
+    if (use_sk) {
+        const int sp = gemm_skinny_splits(md.q_dim, md.d, c->n_sms);
+        SkinnyArgs ga{};
+        ga.R = R; ga.N = md.q_dim; ga.K = md.d; ga.out_f32 = sk; ga.split_stride = (int64_t)R * md.q_dim;
+        ga.ldo = md.q_dim;
+        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WQ][l], nullptr, ga, sp, c->d_status, s);
+        if (st != KVR_OK) return st;
+        launch_rope_scatter(false, sk, md.q_dim, cs, cm, q_only, c->av, l, true, q, ex, s, sp, ga.split_stride);
+    } else if (use_tc_q) {
         TcGemmEpilogue ep{};
         set_tc_extras(ep, ex, true);
         ep.mode = TC_QKV; ep.M = R; ep.K = md.d; ep.N = md.q_dim;
@@ -1033,8 +1059,6 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     } else {
         float *tmp = (float *)m;
         launch_gemm_simt(fp32, 0, a, md.d, c->w[W_WQ][l], nullptr, md.d, R, md.q_dim, md.d, tmp, md.q_dim, s);
-        ModelDims q_only = md;
-        q_only.Hkv = 0; q_only.kv_dim = 0;
         launch_rope_scatter(fp32, tmp, md.q_dim, cs, cm, q_only, c->av, l, true, q, ex, s);
     }
     // one query row per request: the split-KV kernel reads each request's K/V once (bf16, groups of up to 8 heads)
@@ -1055,6 +1079,34 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         if (st != KVR_OK) return st;
     } else {
         launch_attn_simt(fp32, q, cm, d_tables, width, md, c->av, l, a, s);
+    }
+    if (use_sk) {
+        // output projection -> h = h0 + o Wo^T, norm; SwiGLU pair; down projection -> h += ..., final norm; head
+        const int64_t hs = (int64_t)R * md.d;
+        int sp = gemm_skinny_splits(md.d, md.q_dim, c->n_sms);
+        SkinnyArgs go{};
+        go.R = R; go.N = md.d; go.K = md.q_dim; go.out_f32 = sk; go.split_stride = hs; go.ldo = md.d;
+        st = launch_gemm_skinny(c->tm_la_q, c->tm_w[W_WO][l], nullptr, go, sp, c->d_status, s);
+        if (st != KVR_OK) return st;
+        launch_add_rmsnorm(false, h0, h, sk, sp, hs, c->w[W_LN2][l], a, R, md.d, md.eps, s);
+        SkinnyArgs gg{};
+        gg.R = R; gg.N = md.F; gg.K = md.d; gg.out_bf16 = (__nv_bfloat16 *)m; gg.ld_bf16 = md.F;
+        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WG][l], &c->tm_w[W_WU][l], gg, 1, c->d_status, s);
+        if (st != KVR_OK) return st;
+        sp = gemm_skinny_splits(md.d, md.F, c->n_sms);
+        SkinnyArgs gd{};
+        gd.R = R; gd.N = md.d; gd.K = md.F; gd.out_f32 = sk; gd.split_stride = hs; gd.ldo = md.d;
+        st = launch_gemm_skinny(c->tm_lm, c->tm_w[W_WD][l], nullptr, gd, sp, c->d_status, s);
+        if (st != KVR_OK) return st;
+        launch_add_rmsnorm(false, h, h, sk, sp, hs, final_gain, a, R, md.d, md.eps, s);
+        CUtensorMap tlm;
+        st = tc_make_tmap_2d(&tlm, lm_head, md.V, md.d, 128, 64);
+        if (st != KVR_OK) return st;
+        SkinnyArgs gl{};
+        gl.R = R; gl.N = md.V; gl.K = md.d; gl.out_f32 = logits_out; gl.split_stride = 0; gl.ldo = md.V;
+        st = launch_gemm_skinny(c->tm_la_d, tlm, nullptr, gl, 1, c->d_status, s);
+        if (st != KVR_OK) return st;
+        return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
     }
     if (use_tc) {
         TcGemmEpilogue ep{};

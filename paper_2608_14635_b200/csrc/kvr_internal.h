@@ -54,10 +54,11 @@ void launch_embed_rmsnorm(bool fp32, const void *embed, const void *gain, const 
                           void *a, int d, float eps, cudaStream_t s);
 void launch_rmsnorm(bool fp32, const float *h, const void *gain, void *a, int n, int d, float eps,
                     cudaStream_t s);
-// h += part (both fp32 [n, d]), then a = rmsnorm(h) * gain: the residual add of a tensor-parallel partial sum
-// folded into the norm that follows it
-void launch_add_rmsnorm(bool fp32, float *h, const float *part, const void *gain, void *a, int n, int d, float eps,
-                        cudaStream_t s);
+// h_out = h_in + part[0] + ... + part[n_part - 1] (all fp32 [n, d], partial products part_stride elements apart;
+// h_out may be h_in), then a = rmsnorm(h_out) * gain: the residual add of a row-parallel projection's partial
+// sums folded into the norm that follows it
+void launch_add_rmsnorm(bool fp32, const float *h_in, float *h_out, const float *part, int n_part,
+                        int64_t part_stride, const void *gain, void *a, int n, int d, float eps, cudaStream_t s);
 void launch_rope_table(const int32_t *pos, int n, int hd, const RopeFreq &f, float2 *cs, cudaStream_t s);
 // mode 0: C fp32 [M, ldc] = A W0^T; 1: C fp32 += A W0^T; 2: C (T) = silu(A W0^T) * (A W1^T)
 void launch_gemm_simt(bool fp32, int mode, const void *A, int lda, const void *W0, const void *W1, int ldw,
@@ -70,10 +71,11 @@ struct QkvExtras {
     float eps = 0.f;
     bool any() const { return bq || bk || bv || qn || kn; }
 };
-// Reads raw fp32 [n, q_dim + 2 kv_dim] projections; writes rotated Q (T) and the arena rows.
+// Reads raw fp32 [n, q_dim + 2 kv_dim] projections (the sum of n_part partial products part_stride
+// elements apart); writes rotated Q (T) and the arena rows.
 void launch_rope_scatter(bool fp32, const float *qkv, int ld, const float2 *cs, const ChunkMeta &cm,
                          const ModelDims &md, const ArenaView &av, int layer, bool want_q, void *q_out,
-                         const QkvExtras &ex, cudaStream_t s);
+                         const QkvExtras &ex, cudaStream_t s, int n_part = 1, int64_t part_stride = 0);
 void launch_attn_simt(bool fp32, const void *q, const ChunkMeta &cm, const int32_t *tables, int max_blk,
                       const ModelDims &md, const ArenaView &av, int layer, void *o, cudaStream_t s);
 void launch_gather_rows(const float *h, int d, const int2 *pairs, int n_pairs, float *h_last, cudaStream_t s);
@@ -114,6 +116,22 @@ int tc_make_tmap_f32(CUtensorMap *out, const void *base, int64_t rows, int64_t c
 // pair: run on CTA pairs (256 x 256 tiles, tcgen05 cta_group::2) instead of single CTAs
 int launch_gemm_tc(const CUtensorMap &tmA, const CUtensorMap *tmB /*[3]*/, const TcGemmEpilogue &ep,
                    int *d_status, int n_sms, cudaStream_t s, const CUtensorMap *tmH = nullptr, bool pair = false);
+
+// ---- weight-streaming GEMM for the few rows of kv_resume_logits (kvr_gemm_skinny.cu) ----
+constexpr int GEMM_SKINNY_MAX_ROWS = 128, GEMM_SKINNY_MAX_SPLITS = 8;
+struct SkinnyArgs {
+    int R, N, K;              // out[r, n] = sum_k X[r, k] W[n, k], r < R <= 128
+    float *out_f32;           // plain: partial product of split s at out_f32 + s * split_stride, row stride ldo
+    int64_t split_stride;
+    int ldo;
+    __nv_bfloat16 *out_bf16;  // SwiGLU pair (two weight maps): silu(X Wg^T) * (X Wu^T), row stride ld_bf16
+    int ld_bf16;
+};
+int gemm_skinny_init(int device);
+int gemm_skinny_splits(int N, int K, int n_sms);
+// tmX: activation map (box 128 rows x 64), tmW0 / tmW1: weight maps (box 128 x 64); tmW1 non-null = SwiGLU pair
+int launch_gemm_skinny(const CUtensorMap &tmX, const CUtensorMap &tmW0, const CUtensorMap *tmW1,
+                       const SkinnyArgs &a, int splits, int *d_status, cudaStream_t s);
 
 // ---- tensor-core attention (kvr_attn_tc.cu) ----
 int attn_tc_init(int device);

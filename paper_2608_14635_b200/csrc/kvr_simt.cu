@@ -148,22 +148,26 @@ __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restric
     }
 }
 
-// h += part, then the norm of the updated row (tensor-parallel ranks: `part` is the all-reduced
-// partial product of the preceding row-parallel projection).
+// h_out = h_in + sum of n_part partial products (summed in index order), then the norm of the
+// updated row.  Partial products come from the row-parallel projection of a tensor-parallel rank
+// (one, already all-reduced) or from the K splits of the weight-streaming GEMM.
 template <typename T>
-__global__ void __launch_bounds__(256) add_rmsnorm_kernel(float *__restrict__ h, const float *__restrict__ part,
-                                                          const T *__restrict__ gain, T *__restrict__ a, int d,
-                                                          float eps) {
+__global__ void __launch_bounds__(256) add_rmsnorm_kernel(const float *__restrict__ h_in, float *__restrict__ h_out,
+                                                          const float *__restrict__ part, int n_part,
+                                                          int64_t part_stride, const T *__restrict__ gain,
+                                                          T *__restrict__ a, int d, float eps) {
     constexpr int VEC = sizeof(T) == 4 ? 4 : 8;
     extern __shared__ float row[];
     __shared__ float red[32];
     const int64_t t = blockIdx.x;
     float ss = 0.f;
     for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-        float4 x = *reinterpret_cast<const float4 *>(h + t * d + i);
-        const float4 y = *reinterpret_cast<const float4 *>(part + t * d + i);
-        x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
-        *reinterpret_cast<float4 *>(h + t * d + i) = x;
+        float4 x = *reinterpret_cast<const float4 *>(h_in + t * d + i);
+        for (int p = 0; p < n_part; ++p) {
+            const float4 y = *reinterpret_cast<const float4 *>(part + p * part_stride + t * d + i);
+            x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+        }
+        *reinterpret_cast<float4 *>(h_out + t * d + i) = x;
         *reinterpret_cast<float4 *>(row + i) = x;
         ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
     }
@@ -178,15 +182,16 @@ __global__ void __launch_bounds__(256) add_rmsnorm_kernel(float *__restrict__ h,
     }
 }
 
-void launch_add_rmsnorm(bool fp32, float *h, const float *part, const void *gain, void *a, int n, int d, float eps,
-                        cudaStream_t s) {
+void launch_add_rmsnorm(bool fp32, const float *h_in, float *h_out, const float *part, int n_part,
+                        int64_t part_stride, const void *gain, void *a, int n, int d, float eps, cudaStream_t s) {
     if (n == 0) return;
     const size_t sm = (size_t)d * sizeof(float);
     if (fp32)
-        add_rmsnorm_kernel<float><<<n, 256, sm, s>>>(h, part, (const float *)gain, (float *)a, d, eps);
+        add_rmsnorm_kernel<float><<<n, 256, sm, s>>>(h_in, h_out, part, n_part, part_stride, (const float *)gain,
+                                                     (float *)a, d, eps);
     else
-        add_rmsnorm_kernel<__nv_bfloat16><<<n, 256, sm, s>>>(h, part, (const __nv_bfloat16 *)gain,
-                                                              (__nv_bfloat16 *)a, d, eps);
+        add_rmsnorm_kernel<__nv_bfloat16><<<n, 256, sm, s>>>(h_in, h_out, part, n_part, part_stride,
+                                                              (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)a, d, eps);
 }
 
 void launch_embed_rmsnorm(bool fp32, const void *embed, const void *gain, const ChunkMeta &cm, float *h,
@@ -336,14 +341,20 @@ void launch_gemm_simt(bool fp32, int mode, const void *A, int lda, const void *W
 // arena rows at slot[t].
 // ---------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restrict__ qkv, int ld,
-                                                           const float2 *__restrict__ cs,
+__global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restrict__ qkv, int ld, int n_part,
+                                                           int64_t part_stride, const float2 *__restrict__ cs,
                                                            const int32_t *__restrict__ slot, int Hq, int Hkv, int hd,
                                                            T *__restrict__ arena_k, int64_t kv_stride,
                                                            bool want_q, T *__restrict__ q_out, QkvExtras ex) {
     const int64_t t = blockIdx.x;
     const int half = hd >> 1;
-    const float *src = qkv + t * ld;
+    const float *src0 = qkv + t * ld;
+    // the projection may arrive as n_part partial products (K splits), summed here in index order
+    auto src = [&](int i) {
+        float v = src0[i];
+        for (int p = 1; p < n_part; ++p) v += src0[p * part_stride + i];
+        return v;
+    };
     const float2 *c = cs + t * half;
     const int q_dim = Hq * hd, kv_dim = Hkv * hd;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -360,8 +371,8 @@ __global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restri
             const int i = lane + 32 * e;
             x1[e] = x2[e] = 0.f;
             if (i < half) {
-                x1[e] = src[hh * hd + i] + (bias ? to_f<T>(bias[i]) : 0.f);
-                x2[e] = src[hh * hd + i + half] + (bias ? to_f<T>(bias[i + half]) : 0.f);
+                x1[e] = src(hh * hd + i) + (bias ? to_f<T>(bias[i]) : 0.f);
+                x2[e] = src(hh * hd + i + half) + (bias ? to_f<T>(bias[i + half]) : 0.f);
                 ss += x1[e] * x1[e] + x2[e] * x2[e];
             }
         }
@@ -391,21 +402,21 @@ __global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restri
     if (kv_dim > 0) {
         T *vrow = arena_k + (int64_t)slot[t] * kv_dim + kv_stride;
         for (int idx = threadIdx.x; idx < kv_dim; idx += blockDim.x)
-            vrow[idx] = from_f<T>(src[q_dim + kv_dim + idx] + (bv ? to_f<T>(bv[idx]) : 0.f));
+            vrow[idx] = from_f<T>(src(q_dim + kv_dim + idx) + (bv ? to_f<T>(bv[idx]) : 0.f));
     }
 }
 
 void launch_rope_scatter(bool fp32, const float *qkv, int ld, const float2 *cs, const ChunkMeta &cm,
                          const ModelDims &md, const ArenaView &av, int layer, bool want_q, void *q_out,
-                         const QkvExtras &ex, cudaStream_t s) {
+                         const QkvExtras &ex, cudaStream_t s, int n_part, int64_t part_stride) {
     if (cm.n == 0) return;
     if (fp32) {
         float *ak = (float *)av.base + (int64_t)layer * av.layer_stride;
-        rope_scatter_kernel<float><<<cm.n, 128, 0, s>>>(qkv, ld, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak, av.kv_stride,
+        rope_scatter_kernel<float><<<cm.n, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak, av.kv_stride,
                                                          want_q, (float *)q_out, ex);
     } else {
         __nv_bfloat16 *ak = (__nv_bfloat16 *)av.base + (int64_t)layer * av.layer_stride;
-        rope_scatter_kernel<__nv_bfloat16><<<cm.n, 128, 0, s>>>(qkv, ld, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak,
+        rope_scatter_kernel<__nv_bfloat16><<<cm.n, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak,
                                                                  av.kv_stride, want_q, (__nv_bfloat16 *)q_out, ex);
     }
 }

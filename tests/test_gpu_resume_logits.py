@@ -86,7 +86,8 @@ def test_resume_logits_with_fully_shared_request():
     compare_rebuilt(rig, batch, kv, 1e-4, 1e-3)
 
 
-def test_mid_shape_resume_logits():
+@pytest.mark.parametrize("resume_gemm", [1, 0])
+def test_mid_shape_resume_logits(resume_gemm):
     shape = ModelShape("mid", 4, 1024, 8, 2, 128, 2816, 4096)
     spec = dataclasses.replace(WORKLOADS["cfg2"], n_requests=4, fixed_lens=(300, 1000, 77, 2049),
                                lognormal_median=None, clip=None, seed=21)
@@ -95,6 +96,36 @@ def test_mid_shape_resume_logits():
     rig = Rig(shape, "bf16", wl.num_blocks, max_chunk=2048, max_requests=8,
               max_blocks_per_req=batch.tables.shape[1], seed=21)
     assert rig.ctx.kv_set_option("keep_last_hidden", 1) == 0
+    assert rig.ctx.kv_set_option("resume_gemm", resume_gemm) == 0
     rig.rebuild(batch)
     print("mid bf16 logits worst rel-L2", _check(rig, batch, 3e-2))
+    assert rig.guards_ok()
+
+
+@pytest.mark.parametrize("resume_gemm", [1, 0])
+def test_resume_logits_many_requests_ragged_head_and_repeat(resume_gemm):
+    """37 requests (the request dimension is padded to 48 on the tensor core), a vocabulary that ends
+    inside a 128-row weight tile, and the call made twice after one rebuild: the rows the rebuild
+    kept are only read, so both calls give the same bits."""
+    shape = ModelShape("mid-ragged", 2, 1024, 8, 2, 128, 2816, 4100)
+    rng = np.random.default_rng(8)
+    lens = tuple(int(x) for x in rng.integers(1, 260, 37))
+    spec = dataclasses.replace(WORKLOADS["cfg2"], n_requests=37, fixed_lens=lens, lognormal_median=None, clip=None,
+                               seed=23)
+    wl = make_workload(spec, vocab=shape.vocab)
+    batch = wl.rebuild_batch()
+    rig = Rig(shape, "bf16", wl.num_blocks, max_chunk=2048, max_requests=40,
+              max_blocks_per_req=batch.tables.shape[1], seed=23)
+    assert rig.ctx.kv_set_option("keep_last_hidden", 1) == 0
+    assert rig.ctx.kv_set_option("resume_gemm", resume_gemm) == 0
+    rig.rebuild(batch)
+    print("37 requests, logits worst rel-L2", _check(rig, batch, 3e-2))
+    gain, lm = _head(shape, rig.tdtype, rig.dev)
+    outs = []
+    for _ in range(2):
+        out = torch.full((37, shape.vocab), float("nan"), device=rig.dev)
+        assert rig.ctx.kv_resume_logits(gain, lm, out) == 0
+        assert rig.ctx.kv_sync_status() == 0
+        outs.append(out.cpu())
+    assert torch.equal(outs[0], outs[1])
     assert rig.guards_ok()

@@ -7,6 +7,7 @@ import time
 
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from synth import MODEL_SHAPES, WORKLOADS, make_workload
@@ -44,3 +45,40 @@ def test_kernel_waits_run_out_and_are_reported(gemm):
     compare_rebuilt(rig, batch, kv, 1e-2, 6e-2)
     check_untouched(rig, before, batch)
     assert kb.STATUS[rig.ctx.kv_set_option("wait_limit_ms", 60001)] == "KVR_ERR_INVALID_ARG"
+
+
+def test_resume_gemm_waits_run_out_and_are_reported():
+    """The weight-streaming GEMM of kv_resume_logits under the same hook: its waits run out, the call
+    is reported as timed out, and the same call succeeds once the loads are back."""
+    shape = MODEL_SHAPES["tiny"]
+    wl = make_workload(WORKLOADS["cfg1"])
+    batch = wl.rebuild_batch()
+    rig = Rig(shape, "bf16", wl.num_blocks, max_chunk=512, max_requests=8, max_blocks_per_req=batch.tables.shape[1])
+    rig.set_impl(2, 2)
+    assert rig.ctx.kv_set_option("keep_last_hidden", 1) == 0
+    rig.rebuild(batch)
+    g = torch.Generator().manual_seed(5)
+    gain = (1.0 + 0.02 * torch.randn(shape.d_model, generator=g)).to(rig.tdtype).to(rig.dev)
+    lm = (0.02 * torch.randn(shape.vocab, shape.d_model, generator=g)).to(rig.tdtype).to(rig.dev)
+    R = len(batch.lens)
+    good = torch.zeros(R, shape.vocab, device=rig.dev)
+    assert rig.ctx.kv_resume_logits(gain, lm, good) == 0
+    assert rig.ctx.kv_sync_status() == 0
+    before = rig.arena_bits()
+    assert rig.ctx.kv_set_option("wait_limit_ms", 20) == 0
+    assert rig.ctx.kv_set_option("mute_loads", 1) == 0
+    out = torch.zeros(R, shape.vocab, device=rig.dev)
+    t0 = time.perf_counter()
+    assert rig.ctx.kv_resume_logits(gain, lm, out) == 0
+    st = rig.ctx.kv_sync_status()
+    dt = time.perf_counter() - t0
+    assert rig.kb.STATUS[st] == "KVR_ERR_DEVICE_TIMEOUT"
+    assert dt < 2.0, dt
+    assert rig.ctx.kv_set_option("mute_loads", 0) == 0
+    assert rig.ctx.kv_set_option("wait_limit_ms", 0) == 0
+    assert rig.ctx.kv_sync_status() == 0
+    assert rig.ctx.kv_resume_logits(gain, lm, out) == 0
+    assert rig.ctx.kv_sync_status() == 0
+    assert torch.equal(out, good)
+    assert np.array_equal(rig.arena_bits(), before)
+    assert rig.guards_ok()
