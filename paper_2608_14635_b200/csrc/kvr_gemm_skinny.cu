@@ -6,11 +6,13 @@
 //     the MMA's M, the requests are its N (padded to a multiple of 16), so the accumulator
 //     in TMEM is out^T: lane = weight row n, column = request r, and a warp's store of one
 //     column writes 32 consecutive n of one output row;
-//   - one tile per CTA, grid (ceil(N / 128), splits); a split covers a contiguous range of
-//     64-wide K blocks and writes its fp32 partial product to out + split * split_stride,
-//     which the consumer kernel sums in a fixed order (no atomics, run-to-run identical);
-//   - a TMA ring of six 32 KB stages (four 48 KB stages for the SwiGLU pair) keeps about
-//     100 KB of weight bytes in flight per SM.
+//   - a work item is (128-row tile, split); a split covers a contiguous range of 64-wide K
+//     blocks and writes its fp32 partial product to out + split * split_stride, which the
+//     consumer kernel sums in a fixed order (no atomics, run-to-run identical);
+//   - persistent CTAs, one per SM, take items round-robin; a TMA ring of six 32 KB stages
+//     (four 48 KB stages for the SwiGLU pair) keeps about 100 KB of weight bytes in flight
+//     per SM across items, and two accumulator buffers in TMEM let the epilogue of one item
+//     run under the loads and MMAs of the next.
 // Warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue.
 // Every wait is bounded through the context's status block, as in the large GEMM.
 #include "kvr_internal.h"
@@ -29,20 +31,34 @@ struct SkCfg {
     static constexpr int STAGES = SWIGLU ? 4 : 6;
     static constexpr int N_W = SWIGLU ? 2 : 1;                       // weight boxes per stage
     static constexpr int STAGE_BYTES = (N_W + 1) * SK_TILE_BYTES;    // weights, then the activation box
-    static constexpr int TMEM_COLS = SWIGLU ? 256 : 128;
+    static constexpr int ACC_COLS = SWIGLU ? 256 : 128;              // one accumulator buffer (gate | up)
+    static constexpr int TMEM_COLS = 2 * ACC_COLS;                   // two buffers: epilogue overlaps the next item
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
 };
+
+// Work item w of a launch: tile = w % n_tiles, split = w / n_tiles (neighbouring CTAs share a K range of X).
+struct SkItem { int tile, kb0, kb1; int split; };
+__device__ __forceinline__ SkItem sk_item(int w, int n_tiles, int n_split, int num_k) {
+    SkItem it;
+    it.split = w / n_tiles;
+    it.tile = w - it.split * n_tiles;
+    it.kb0 = (int)((int64_t)it.split * num_k / n_split);
+    it.kb1 = (int)((int64_t)(it.split + 1) * num_k / n_split);
+    return it;
+}
 
 template <bool SWIGLU>
 __global__ void __launch_bounds__(SK_THREADS, 1)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
-                   const __grid_constant__ CUtensorMap tmW1, const SkinnyArgs a, int *status) {
+                   const __grid_constant__ CUtensorMap tmW1, const SkinnyArgs a, int n_split, int *status) {
     using Cfg = SkCfg<SWIGLU>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t bars = tiles + Cfg::STAGES * Cfg::STAGE_BYTES;
-    const uint32_t full0 = bars, empty0 = bars + 8 * Cfg::STAGES, tfull = bars + 16 * Cfg::STAGES;
+    // barrier addresses: full[s], empty[s], tmem_full[2], tmem_empty[2]
+    const uint32_t full0 = bars, empty0 = bars + 8 * Cfg::STAGES, tfull0 = bars + 16 * Cfg::STAGES,
+                   tempty0 = bars + 16 * Cfg::STAGES + 16;
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
 
@@ -53,7 +69,10 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             ptx::mbar_init(full0 + 8 * s, 1);
             ptx::mbar_init(empty0 + 8 * s, 1);
         }
-        ptx::mbar_init(tfull, 1);
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull0 + 8 * b, 1);
+            ptx::mbar_init(tempty0 + 8 * b, 4);
+        }
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmX);
         ptx::prefetch_tmap(&tmW0);
@@ -68,61 +87,78 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const uint32_t tmem_base = tmem_base_sh;
     volatile int *abort_flag = &abort_sh;
 
-    const int tile = blockIdx.x, split = blockIdx.y, n_split = gridDim.y;
+    const int n_tiles = (a.N + SK_ROWS - 1) / SK_ROWS;
+    const int total = n_tiles * n_split;
     const int num_k = (a.K + SK_BK - 1) / SK_BK;
-    const int kb0 = (int)((int64_t)split * num_k / n_split), kb1 = (int)((int64_t)(split + 1) * num_k / n_split);
-    const bool empty = kb1 <= kb0;   // more splits than K blocks: this split's partial product is zero
     const int n_pad = a.R <= 16 ? 16 : ((a.R + 15) & ~15);
+    // a split with no K block (more splits than blocks) has a zero partial product: the producer and the MMA
+    // thread skip the item, the epilogue stores zeros without touching an accumulator
 
     if (warp == 0) {
-        if (lane == 0 && !empty && !ptx::loads_muted(status)) {
-            int stage = 0;
-            uint32_t phase = 0;
-            for (int kb = kb0; kb < kb1; ++kb) {
-                if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1u, status, abort_flag)) break;
-                const uint32_t fb = full0 + 8 * stage;
-                const uint32_t sa = tiles + stage * Cfg::STAGE_BYTES;
-                ptx::mbar_expect_tx(fb, Cfg::STAGE_BYTES);
-                ptx::tma_load_2d(sa, &tmW0, kb * SK_BK, tile * SK_ROWS, fb);
-                if (SWIGLU) ptx::tma_load_2d(sa + SK_TILE_BYTES, &tmW1, kb * SK_BK, tile * SK_ROWS, fb);
-                ptx::tma_load_2d(sa + Cfg::N_W * SK_TILE_BYTES, &tmX, kb * SK_BK, 0, fb);
-                if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0 && !empty) {
-            const uint32_t idesc = ptx::idesc_bf16(SK_ROWS, n_pad);
+        if (lane == 0 && !ptx::loads_muted(status)) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int kb = kb0; kb < kb1; ++kb) {
-                if (!ptx::mbar_wait(full0 + 8 * stage, phase, status, abort_flag)) { ok = false; break; }
-                ptx::tc_fence_after();
-                const uint32_t sa = tiles + stage * Cfg::STAGE_BYTES;
-                const uint64_t dw0 = ptx::smem_desc_sw128(sa);
-                const uint64_t dw1 = ptx::smem_desc_sw128(sa + SK_TILE_BYTES);
-                const uint64_t dx = ptx::smem_desc_sw128(sa + Cfg::N_W * SK_TILE_BYTES);
-#pragma unroll
-                for (int kk = 0; kk < SK_BK / SK_UMMA_K; ++kk) {
-                    const uint32_t accum = (kb > kb0 || kk > 0) ? 1u : 0u;
-                    ptx::mma_bf16_ss(tmem_base, dw0 + 2 * kk, dx + 2 * kk, idesc, accum);
-                    if (SWIGLU) ptx::mma_bf16_ss(tmem_base + 128, dw1 + 2 * kk, dx + 2 * kk, idesc, accum);
+            for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+                const SkItem it = sk_item(w, n_tiles, n_split, num_k);
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!ptx::mbar_wait(empty0 + 8 * stage, phase ^ 1u, status, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = full0 + 8 * stage;
+                    const uint32_t sa = tiles + stage * Cfg::STAGE_BYTES;
+                    ptx::mbar_expect_tx(fb, Cfg::STAGE_BYTES);
+                    ptx::tma_load_2d(sa, &tmW0, kb * SK_BK, it.tile * SK_ROWS, fb);
+                    if (SWIGLU) ptx::tma_load_2d(sa + SK_TILE_BYTES, &tmW1, kb * SK_BK, it.tile * SK_ROWS, fb);
+                    ptx::tma_load_2d(sa + Cfg::N_W * SK_TILE_BYTES, &tmX, kb * SK_BK, 0, fb);
+                    if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
                 }
-                ptx::mma_commit(empty0 + 8 * stage);
-                if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
             }
-            if (ok) ptx::mma_commit(tfull);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = ptx::idesc_bf16(SK_ROWS, n_pad);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+                const SkItem it = sk_item(w, n_tiles, n_split, num_k);
+                if (it.kb1 <= it.kb0) continue;
+                if (!ptx::mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, status, abort_flag)) break;
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * Cfg::ACC_COLS;
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!ptx::mbar_wait(full0 + 8 * stage, phase, status, abort_flag)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t sa = tiles + stage * Cfg::STAGE_BYTES;
+                    const uint64_t dw0 = ptx::smem_desc_sw128(sa);
+                    const uint64_t dw1 = ptx::smem_desc_sw128(sa + SK_TILE_BYTES);
+                    const uint64_t dx = ptx::smem_desc_sw128(sa + Cfg::N_W * SK_TILE_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < SK_BK / SK_UMMA_K; ++kk) {
+                        const uint32_t accum = (kb > it.kb0 || kk > 0) ? 1u : 0u;
+                        ptx::mma_bf16_ss(d_tmem, dw0 + 2 * kk, dx + 2 * kk, idesc, accum);
+                        if (SWIGLU) ptx::mma_bf16_ss(d_tmem + 128, dw1 + 2 * kk, dx + 2 * kk, idesc, accum);
+                    }
+                    ptx::mma_commit(empty0 + 8 * stage);
+                    if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                ptx::mma_commit(tfull0 + 8 * acc);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
         }
     } else {
         const int quarter = warp & 3;   // the 32 TMEM lanes this warp may read
-        const int n = tile * SK_ROWS + quarter * 32 + lane;
-        bool ok = true;
-        if (!empty) {
-            ok = ptx::mbar_wait(tfull, 0, status, abort_flag);
-            ptx::tc_fence_after();
-        }
-        if (ok) {
-            const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int w = blockIdx.x; w < total; w += gridDim.x) {
+            const SkItem it = sk_item(w, n_tiles, n_split, num_k);
+            const bool empty = it.kb1 <= it.kb0;
+            const int n = it.tile * SK_ROWS + quarter * 32 + lane;
+            if (!empty) {
+                if (!ptx::mbar_wait(tfull0 + 8 * acc, acc_phase, status, abort_flag)) break;
+                ptx::tc_fence_after();
+            }
+            const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * Cfg::ACC_COLS;
 #pragma unroll 1
             for (int c = 0; c < n_pad; c += 16) {
                 uint32_t g[16], u[16];
@@ -147,12 +183,18 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         }
                     }
                 } else {
-                    float *dst = a.out_f32 + (int64_t)split * a.split_stride + n;
+                    float *dst = a.out_f32 + (int64_t)it.split * a.split_stride + n;
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (c + j < a.R) dst[(int64_t)(c + j) * a.ldo] = __uint_as_float(g[j]);
                 }
                 __syncwarp();
+            }
+            if (!empty) {
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(tempty0 + 8 * acc);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
     }
@@ -186,15 +228,19 @@ int gemm_skinny_splits(int N, int K, int n_sms) {
 }
 
 int launch_gemm_skinny(const CUtensorMap &tmX, const CUtensorMap &tmW0, const CUtensorMap *tmW1,
-                       const SkinnyArgs &a, int splits, int *d_status, cudaStream_t s) {
+                       const SkinnyArgs &a, int splits, int *d_status, int n_sms, cudaStream_t s) {
     if (a.R <= 0 || a.N <= 0) return KVR_OK;
     if (a.R > GEMM_SKINNY_MAX_ROWS || a.K <= 0 || splits < 1 || splits > GEMM_SKINNY_MAX_SPLITS)
         return KVR_ERR_UNSUPPORTED;
-    const dim3 grid((a.N + SK_ROWS - 1) / SK_ROWS, tmW1 ? 1 : splits);
+    const int n_split = tmW1 ? 1 : splits;   // the SwiGLU pair needs whole sums before its nonlinearity
+    const int total = (a.N + SK_ROWS - 1) / SK_ROWS * n_split;
+    const int grid = total < n_sms ? total : n_sms;
     if (tmW1)
-        gemm_skinny_kernel<true><<<grid, SK_THREADS, SkCfg<true>::SMEM_BYTES, s>>>(tmX, tmW0, *tmW1, a, d_status);
+        gemm_skinny_kernel<true><<<grid, SK_THREADS, SkCfg<true>::SMEM_BYTES, s>>>(tmX, tmW0, *tmW1, a, n_split,
+                                                                                   d_status);
     else
-        gemm_skinny_kernel<false><<<grid, SK_THREADS, SkCfg<false>::SMEM_BYTES, s>>>(tmX, tmW0, tmW0, a, d_status);
+        gemm_skinny_kernel<false><<<grid, SK_THREADS, SkCfg<false>::SMEM_BYTES, s>>>(tmX, tmW0, tmW0, a, n_split,
+                                                                                     d_status);
     return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
 }
 

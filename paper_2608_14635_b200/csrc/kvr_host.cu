@@ -233,6 +233,25 @@ struct SetDevice {
     ~SetDevice() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
+// Per-request metadata of kv_resume_logits: [pos R][table row R] and one single-row attention tile per request
+// (longest context first).  Written by the rebuild that keeps the final rows, so the resume call copies nothing.
+static size_t resume_meta_bytes(int R) {
+    return align_up((size_t)R * 2 * sizeof(int32_t)) + align_up((size_t)R * sizeof(AttnTile));
+}
+static int upload_resume_meta(kvr_ctx *c, char *staging, const int32_t *lens, int R, cudaStream_t s) {
+    int32_t *st_pos = (int32_t *)staging;
+    AttnTile *st_tiles = (AttnTile *)(staging + align_up((size_t)R * 2 * sizeof(int32_t)));
+    for (int r = 0; r < R; ++r) {
+        st_pos[r] = lens[r] - 1;
+        st_pos[R + r] = r;
+        st_tiles[r] = AttnTile{r, lens[r] - 1, 1, r};
+    }
+    std::stable_sort(st_tiles, st_tiles + R, [](const AttnTile &x, const AttnTile &y) { return x.pos0 > y.pos0; });
+    CU_OK(cudaMemcpyAsync(c->ws + c->lay.l_pos, st_pos, (size_t)R * 2 * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(c->ws + c->lay.l_tiles, st_tiles, (size_t)R * sizeof(AttnTile), cudaMemcpyHostToDevice, s));
+    return KVR_OK;
+}
+
 int ensure_staging(kvr_ctx *c, size_t bytes) {
     if (c->staging_busy) {
         CU_OK(cudaEventSynchronize(c->staging_free));
@@ -677,7 +696,9 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     const size_t meta_bytes = (size_t)T * 4 * sizeof(int32_t);
     const size_t max_tiles_total = (size_t)(T / ATTN_TILE_Q + R + n_chunks + 1);
     const size_t tiles_bytes = align_up(max_tiles_total * sizeof(AttnTile));
-    const size_t stage_bytes = align_up(tables_bytes) + align_up(meta_bytes) + tiles_bytes + (size_t)R * sizeof(int2);
+    const size_t pairs_bytes = align_up((size_t)R * sizeof(int2));
+    const size_t stage_bytes = align_up(tables_bytes) + align_up(meta_bytes) + tiles_bytes + pairs_bytes +
+                               resume_meta_bytes(R);
     st = ensure_staging(c, stage_bytes);
     if (st != KVR_OK) return st;
     int32_t *st_tables = (int32_t *)c->pinned;
@@ -747,6 +768,14 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     int64_t launches = 0;
 
     CU_OK(cudaMemcpyAsync(d_tables, st_tables, tables_bytes, cudaMemcpyHostToDevice, s));
+    bool all_nonempty = true;
+    for (int r = 0; r < R; ++r) all_nonempty = all_nonempty && lens[r] > 0;
+    if (c->keep_last && all_nonempty) {
+        // what kv_resume_logits needs besides the kept rows goes up with the tables
+        char *st_resume = c->pinned + align_up(tables_bytes) + align_up(meta_bytes) + tiles_bytes + pairs_bytes;
+        st = upload_resume_meta(c, st_resume, lens, R, s);
+        if (st != KVR_OK) return st;
+    }
     for (int64_t k = 0; k < n_chunks; ++k) {
         const Chunk &ch = chunks[k];
         const int n = ch.n;
@@ -900,9 +929,7 @@ int kv_rebuild_from(kvr_ctx *c, const kv_weights *weights, const int32_t *tokens
     c->last_launches = launches;
     c->dev_tables_current = true;
     if (c->keep_last) {
-        bool all = true;
-        for (int r = 0; r < R; ++r) all = all && lens[r] > 0;
-        c->have_last = all;
+        c->have_last = all_nonempty;
         c->last_lens.assign(lens, lens + R);
         c->last_tables.assign(tables, tables + (size_t)R * width);
         c->last_width = width;
@@ -1000,29 +1027,21 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     int32_t *d_pos = (int32_t *)(ws + L.l_pos), *d_row = d_pos + R;
     int32_t *d_tables = (int32_t *)(ws + L.tables);
     AttnTile *d_tiles = (AttnTile *)(ws + L.l_tiles);
-    // per-request metadata: position of the final token, table row, one-row attention tile
-    const size_t tb = (size_t)R * width * sizeof(int32_t);
-    const size_t need = align_up(tb) + align_up((size_t)R * 2 * sizeof(int32_t)) + (size_t)R * sizeof(AttnTile);
-    int st = ensure_staging(c, need);
-    if (st != KVR_OK) return st;
-    int32_t *st_tab = (int32_t *)c->pinned;
-    int32_t *st_pos = (int32_t *)(c->pinned + align_up(tb));
-    AttnTile *st_tiles = (AttnTile *)(c->pinned + align_up(tb) + align_up((size_t)R * 2 * sizeof(int32_t)));
-    // the block tables are still in the workspace when nothing but the rebuild has used it since
-    const bool copy_tables = !c->dev_tables_current;
-    if (copy_tables) std::memcpy(st_tab, c->last_tables.data(), tb);
-    for (int r = 0; r < R; ++r) {
-        st_pos[r] = c->last_lens[r] - 1;
-        st_pos[R + r] = r;
-        st_tiles[r] = AttnTile{r, c->last_lens[r] - 1, 1, r};
+    // the block tables and the per-request metadata are still in the workspace when nothing but the rebuild
+    // has used it since; otherwise they go up again
+    int st = KVR_OK;
+    if (!c->dev_tables_current) {
+        const size_t tb = (size_t)R * width * sizeof(int32_t);
+        st = ensure_staging(c, align_up(tb) + resume_meta_bytes(R));
+        if (st != KVR_OK) return st;
+        std::memcpy(c->pinned, c->last_tables.data(), tb);
+        CU_OK(cudaMemcpyAsync(d_tables, c->pinned, tb, cudaMemcpyHostToDevice, s));
+        st = upload_resume_meta(c, c->pinned + align_up(tb), c->last_lens.data(), R, s);
+        if (st != KVR_OK) return st;
+        CU_OK(cudaEventRecord(c->staging_free, s));
+        c->staging_busy = true;
+        c->dev_tables_current = true;
     }
-    std::stable_sort(st_tiles, st_tiles + R, [](const AttnTile &x, const AttnTile &y) { return x.pos0 > y.pos0; });
-    if (copy_tables) CU_OK(cudaMemcpyAsync(d_tables, st_tab, tb, cudaMemcpyHostToDevice, s));
-    c->dev_tables_current = true;
-    CU_OK(cudaMemcpyAsync(d_pos, st_pos, (size_t)R * 2 * sizeof(int32_t), cudaMemcpyHostToDevice, s));
-    CU_OK(cudaMemcpyAsync(d_tiles, st_tiles, (size_t)R * sizeof(AttnTile), cudaMemcpyHostToDevice, s));
-    CU_OK(cudaEventRecord(c->staging_free, s));
-    c->staging_busy = true;
     RopeFreq rf;
     for (int i = 0; i < md.hd / 2; ++i) rf.inv_freq[i] = std::pow(md.rope_base, -2.0 * i / md.hd);
     ChunkMeta cm{d_pos, d_pos, d_pos, d_row, R};   // tok and slot are not used on this path
@@ -1042,7 +1061,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         SkinnyArgs ga{};
         ga.R = R; ga.N = md.q_dim; ga.K = md.d; ga.out_f32 = sk; ga.split_stride = (int64_t)R * md.q_dim;
         ga.ldo = md.q_dim;
-        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WQ][l], nullptr, ga, sp, c->d_status, s);
+        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WQ][l], nullptr, ga, sp, c->d_status, c->n_sms, s);
         if (st != KVR_OK) return st;
         launch_rope_scatter(false, sk, md.q_dim, cs, cm, q_only, c->av, l, true, q, ex, s, sp, ga.split_stride);
     } else if (use_tc_q) {
@@ -1086,17 +1105,17 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         int sp = gemm_skinny_splits(md.d, md.q_dim, c->n_sms);
         SkinnyArgs go{};
         go.R = R; go.N = md.d; go.K = md.q_dim; go.out_f32 = sk; go.split_stride = hs; go.ldo = md.d;
-        st = launch_gemm_skinny(c->tm_la_q, c->tm_w[W_WO][l], nullptr, go, sp, c->d_status, s);
+        st = launch_gemm_skinny(c->tm_la_q, c->tm_w[W_WO][l], nullptr, go, sp, c->d_status, c->n_sms, s);
         if (st != KVR_OK) return st;
         launch_add_rmsnorm(false, h0, h, sk, sp, hs, c->w[W_LN2][l], a, R, md.d, md.eps, s);
         SkinnyArgs gg{};
         gg.R = R; gg.N = md.F; gg.K = md.d; gg.out_bf16 = (__nv_bfloat16 *)m; gg.ld_bf16 = md.F;
-        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WG][l], &c->tm_w[W_WU][l], gg, 1, c->d_status, s);
+        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WG][l], &c->tm_w[W_WU][l], gg, 1, c->d_status, c->n_sms, s);
         if (st != KVR_OK) return st;
         sp = gemm_skinny_splits(md.d, md.F, c->n_sms);
         SkinnyArgs gd{};
         gd.R = R; gd.N = md.d; gd.K = md.F; gd.out_f32 = sk; gd.split_stride = hs; gd.ldo = md.d;
-        st = launch_gemm_skinny(c->tm_lm, c->tm_w[W_WD][l], nullptr, gd, sp, c->d_status, s);
+        st = launch_gemm_skinny(c->tm_lm, c->tm_w[W_WD][l], nullptr, gd, sp, c->d_status, c->n_sms, s);
         if (st != KVR_OK) return st;
         launch_add_rmsnorm(false, h, h, sk, sp, hs, final_gain, a, R, md.d, md.eps, s);
         CUtensorMap tlm;
@@ -1104,7 +1123,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         if (st != KVR_OK) return st;
         SkinnyArgs gl{};
         gl.R = R; gl.N = md.V; gl.K = md.d; gl.out_f32 = logits_out; gl.split_stride = 0; gl.ldo = md.V;
-        st = launch_gemm_skinny(c->tm_la_d, tlm, nullptr, gl, 1, c->d_status, s);
+        st = launch_gemm_skinny(c->tm_la_d, tlm, nullptr, gl, 1, c->d_status, c->n_sms, s);
         if (st != KVR_OK) return st;
         return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
     }

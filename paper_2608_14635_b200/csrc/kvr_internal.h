@@ -131,7 +131,7 @@ int gemm_skinny_init(int device);
 int gemm_skinny_splits(int N, int K, int n_sms);
 // tmX: activation map (box 128 rows x 64), tmW0 / tmW1: weight maps (box 128 x 64); tmW1 non-null = SwiGLU pair
 int launch_gemm_skinny(const CUtensorMap &tmX, const CUtensorMap &tmW0, const CUtensorMap *tmW1,
-                       const SkinnyArgs &a, int splits, int *d_status, cudaStream_t s);
+                       const SkinnyArgs &a, int splits, int *d_status, int n_sms, cudaStream_t s);
 
 // ---- tensor-core attention (kvr_attn_tc.cu) ----
 int attn_tc_init(int device);

@@ -360,7 +360,8 @@ __global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *bq = (const T *)ex.bq, *bk = (const T *)ex.bk, *bv = (const T *)ex.bv;
     // one warp per q or k head: lane owns pairs i = lane, lane + 32 (hd <= 128)
-    for (int hh = warp; hh < Hq + Hkv; hh += 4) {
+    // blockIdx.y spreads the heads of a row over several blocks (few rows: the resume call)
+    for (int hh = warp + 4 * blockIdx.y; hh < Hq + Hkv; hh += 4 * gridDim.y) {
         const bool is_q = hh < Hq;
         if (is_q && !want_q) continue;
         const T *bias = is_q ? (bq ? bq + hh * hd : nullptr) : (bk ? bk + (hh - Hq) * hd : nullptr);
@@ -401,7 +402,7 @@ __global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restri
     }
     if (kv_dim > 0) {
         T *vrow = arena_k + (int64_t)slot[t] * kv_dim + kv_stride;
-        for (int idx = threadIdx.x; idx < kv_dim; idx += blockDim.x)
+        for (int idx = threadIdx.x + blockDim.x * blockIdx.y; idx < kv_dim; idx += blockDim.x * gridDim.y)
             vrow[idx] = from_f<T>(src(q_dim + kv_dim + idx) + (bv ? to_f<T>(bv[idx]) : 0.f));
     }
 }
@@ -410,13 +411,15 @@ void launch_rope_scatter(bool fp32, const float *qkv, int ld, const float2 *cs, 
                          const ModelDims &md, const ArenaView &av, int layer, bool want_q, void *q_out,
                          const QkvExtras &ex, cudaStream_t s, int n_part, int64_t part_stride) {
     if (cm.n == 0) return;
+    // one block per row when there are rows enough to fill the GPU, else one block per four heads
+    const dim3 grid(cm.n, cm.n >= 1024 ? 1 : (md.Hq + md.Hkv + 3) / 4);
     if (fp32) {
         float *ak = (float *)av.base + (int64_t)layer * av.layer_stride;
-        rope_scatter_kernel<float><<<cm.n, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak, av.kv_stride,
+        rope_scatter_kernel<float><<<grid, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak, av.kv_stride,
                                                          want_q, (float *)q_out, ex);
     } else {
         __nv_bfloat16 *ak = (__nv_bfloat16 *)av.base + (int64_t)layer * av.layer_stride;
-        rope_scatter_kernel<__nv_bfloat16><<<cm.n, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak,
+        rope_scatter_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak,
                                                                  av.kv_stride, want_q, (__nv_bfloat16 *)q_out, ex);
     }
 }
