@@ -325,7 +325,8 @@ int kv_debug_profile(kvr_ctx *ctx, double *ms_by_kind, int64_t *launches_by_kind
  * "attn" 0 = plain kernel, 1 = warp-level MMA kernel, 2 = tcgen05 kernel (1 and 2 bf16 only; 2 is the
  * default in bf16 and needs block_size 16, otherwise 1 is used); "resume_gemm" 0/1 (kv_resume_logits with the tcgen05
  * kernels and at most 128 requests: 1 = projections by the weight-streaming kernel that cuts the grid along the weight rows
- * and K, the default; 0 = by the rebuild's GEMM).
+ * and K, the default; 0 = by the rebuild's GEMM); "resume_overlap" 0/1 (on that path, launch every kernel after the first norm
+ * so that it may be scheduled while the kernel before it drains; it still waits for that kernel's results; default 1).
  * Returns KVR_ERR_INVALID_ARG for unknown names or values. */
 int kv_set_option(kvr_ctx *ctx, const char *name, int64_t value);
 

@@ -60,6 +60,8 @@ attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *_
     constexpr int KP = HD / 32;            // pairs of k-steps of Q K^T
     constexpr int NT = HD / 8;             // 8-dim column tiles of O
     constexpr int ROW_CHUNKS = HD / 8;     // 16-byte chunks per V row
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int sp = blockIdx.x, hk = blockIdx.y, r = blockIdx.z;
     const int G = Hq / Hkv;
     const int n_keys = pos[r] + 1;
@@ -201,6 +203,8 @@ template <int HD>
 __global__ void __launch_bounds__(HD)
 attn_decode_merge_kernel(const float *__restrict__ partial, const int32_t *__restrict__ pos, int Hq, int split_len,
                          int max_splits, __nv_bfloat16 *__restrict__ o) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int hq = blockIdx.x, r = blockIdx.y, d = threadIdx.x;
     const int n_splits = (pos[r] + split_len) / split_len;   // ceil((pos + 1) / split_len)
     const float *base = partial + ((int64_t)r * Hq + hq) * max_splits * (HD + 2);
@@ -223,7 +227,7 @@ size_t attn_decode_scratch_bytes(int max_requests, int Hq, int hd) {
 
 int launch_attn_decode(const __nv_bfloat16 *q, const int32_t *pos, int R, int max_len, const int32_t *tables,
                        int max_blk, const ModelDims &md, const ArenaView &av, int layer, float *scratch,
-                       __nv_bfloat16 *o, cudaStream_t s) {
+                       __nv_bfloat16 *o, cudaStream_t s, bool pdl) {
     if (R <= 0) return KVR_OK;
     if (md.Hq / md.Hkv > DEC_GMAX || (md.hd != 64 && md.hd != 128)) return KVR_ERR_UNSUPPORTED;
     // splits of at least 1024 keys, at most ATTN_DECODE_MAX_SPLITS per request, whole 32-key blocks
@@ -234,15 +238,15 @@ int launch_attn_decode(const __nv_bfloat16 *q, const int32_t *pos, int R, int ma
     const __nv_bfloat16 *ak = (const __nv_bfloat16 *)av.base + (int64_t)layer * av.layer_stride;
     dim3 grid(n_splits, md.Hkv, R), mgrid(md.Hq, R);
     if (md.hd == 128) {
-        attn_decode_partial_kernel<128><<<grid, DEC_THREADS, 0, s>>>(q, pos, tables, max_blk, md.Hq, md.Hkv, ak,
-                                                                     av.kv_stride, av.block_size, split_len,
-                                                                     ATTN_DECODE_MAX_SPLITS, scratch);
-        attn_decode_merge_kernel<128><<<mgrid, 128, 0, s>>>(scratch, pos, md.Hq, split_len, ATTN_DECODE_MAX_SPLITS, o);
+        launch_kernel(attn_decode_partial_kernel<128>, grid, dim3(DEC_THREADS), 0, s, pdl, q, pos, tables, max_blk, md.Hq,
+                      md.Hkv, ak, av.kv_stride, av.block_size, split_len, ATTN_DECODE_MAX_SPLITS, scratch);
+        launch_kernel(attn_decode_merge_kernel<128>, mgrid, dim3(128), 0, s, pdl, (const float *)scratch, pos, md.Hq,
+                      split_len, ATTN_DECODE_MAX_SPLITS, o);
     } else {
-        attn_decode_partial_kernel<64><<<grid, DEC_THREADS, 0, s>>>(q, pos, tables, max_blk, md.Hq, md.Hkv, ak,
-                                                                    av.kv_stride, av.block_size, split_len,
-                                                                    ATTN_DECODE_MAX_SPLITS, scratch);
-        attn_decode_merge_kernel<64><<<mgrid, 64, 0, s>>>(scratch, pos, md.Hq, split_len, ATTN_DECODE_MAX_SPLITS, o);
+        launch_kernel(attn_decode_partial_kernel<64>, grid, dim3(DEC_THREADS), 0, s, pdl, q, pos, tables, max_blk, md.Hq,
+                      md.Hkv, ak, av.kv_stride, av.block_size, split_len, ATTN_DECODE_MAX_SPLITS, scratch);
+        launch_kernel(attn_decode_merge_kernel<64>, mgrid, dim3(64), 0, s, pdl, (const float *)scratch, pos, md.Hq,
+                      split_len, ATTN_DECODE_MAX_SPLITS, o);
     }
     return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
 }

@@ -9,9 +9,10 @@
 //   - a work item is (128-row tile, split); a split covers a contiguous range of 64-wide K
 //     blocks and writes its fp32 partial product to out + split * split_stride, which the
 //     consumer kernel sums in a fixed order (no atomics, run-to-run identical);
-//   - persistent CTAs, one per SM, take items round-robin; a TMA ring of six 32 KB stages
-//     (four 48 KB stages for the SwiGLU pair) keeps about 100 KB of weight bytes in flight
-//     per SM across items, and two accumulator buffers in TMEM let the epilogue of one item
+//   - persistent CTAs, one per SM, take items round-robin; a TMA ring of nine 24 KB stages
+//     (five 40 KB stages for the SwiGLU pair; six and four when there are more than 64
+//     rows) keeps about 150 KB of weight bytes in flight per SM across items - the kernel
+//     is bound by how many bytes it keeps in flight, not by DRAM or L2 throughput - and two accumulator buffers in TMEM let the epilogue of one item
 //     run under the loads and MMAs of the next.
 // Warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue.
 // Every wait is bounded through the context's status block, as in the large GEMM.
@@ -26,11 +27,14 @@ constexpr int SK_ROWS = 128, SK_BK = 64, SK_UMMA_K = 16;
 constexpr int SK_TILE_BYTES = SK_ROWS * SK_BK * 2;   // one 128 x 64 bf16 box
 constexpr int SK_THREADS = 192;
 
-template <bool SWIGLU>
+// XROWS: rows of the activation box (64 when the call has at most 64 rows: the smaller box leaves
+// shared memory for more stages, i.e. more weight bytes in flight)
+template <bool SWIGLU, int XROWS>
 struct SkCfg {
-    static constexpr int STAGES = SWIGLU ? 4 : 6;
     static constexpr int N_W = SWIGLU ? 2 : 1;                       // weight boxes per stage
-    static constexpr int STAGE_BYTES = (N_W + 1) * SK_TILE_BYTES;    // weights, then the activation box
+    static constexpr int X_BYTES = XROWS * SK_BK * 2;
+    static constexpr int STAGE_BYTES = N_W * SK_TILE_BYTES + X_BYTES;   // weights, then the activation box
+    static constexpr int STAGES = (220 * 1024) / STAGE_BYTES;        // 128 rows: 6 / 4 (pair), 64 rows: 9 / 5
     static constexpr int ACC_COLS = SWIGLU ? 256 : 128;              // one accumulator buffer (gate | up)
     static constexpr int TMEM_COLS = 2 * ACC_COLS;                   // two buffers: epilogue overlaps the next item
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
@@ -47,11 +51,11 @@ __device__ __forceinline__ SkItem sk_item(int w, int n_tiles, int n_split, int n
     return it;
 }
 
-template <bool SWIGLU>
+template <bool SWIGLU, int XROWS>
 __global__ void __launch_bounds__(SK_THREADS, 1)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
                    const __grid_constant__ CUtensorMap tmW1, const SkinnyArgs a, int n_split, int *status) {
-    using Cfg = SkCfg<SWIGLU>;
+    using Cfg = SkCfg<SWIGLU, XROWS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -86,6 +90,9 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     ptx::tc_fence_after();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int *abort_flag = &abort_sh;
+    // everything above is local to the CTA and may run while the kernel before this one drains
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     const int n_tiles = (a.N + SK_ROWS - 1) / SK_ROWS;
     const int total = n_tiles * n_split;
@@ -208,14 +215,19 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
 }  // namespace
 
+template <bool SWIGLU, int XROWS>
+static bool sk_set_smem() {
+    return cudaFuncSetAttribute(gemm_skinny_kernel<SWIGLU, XROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                SkCfg<SWIGLU, XROWS>::SMEM_BYTES) == cudaSuccess;
+}
+
 int gemm_skinny_init(int device) {
     (void)device;
-    if (cudaFuncSetAttribute(gemm_skinny_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             SkCfg<false>::SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_skinny_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             SkCfg<true>::SMEM_BYTES) != cudaSuccess)
-        return KVR_ERR_CUDA;
-    return KVR_OK;
+    static_assert(SkCfg<false, 64>::SMEM_BYTES <= 227 * 1024 && SkCfg<true, 64>::SMEM_BYTES <= 227 * 1024 &&
+                  SkCfg<false, 128>::SMEM_BYTES <= 227 * 1024 && SkCfg<true, 128>::SMEM_BYTES <= 227 * 1024, "smem");
+    return sk_set_smem<false, 64>() && sk_set_smem<true, 64>() && sk_set_smem<false, 128>() && sk_set_smem<true, 128>()
+               ? KVR_OK
+               : KVR_ERR_CUDA;
 }
 
 // One wave of CTAs where the matrix has fewer 128-row tiles than the GPU has SMs.
@@ -228,19 +240,32 @@ int gemm_skinny_splits(int N, int K, int n_sms) {
 }
 
 int launch_gemm_skinny(const CUtensorMap &tmX, const CUtensorMap &tmW0, const CUtensorMap *tmW1,
-                       const SkinnyArgs &a, int splits, int *d_status, int n_sms, cudaStream_t s) {
+                       const SkinnyArgs &a, int x_rows, int splits, int *d_status, int n_sms, cudaStream_t s,
+                       bool pdl) {
     if (a.R <= 0 || a.N <= 0) return KVR_OK;
     if (a.R > GEMM_SKINNY_MAX_ROWS || a.K <= 0 || splits < 1 || splits > GEMM_SKINNY_MAX_SPLITS)
         return KVR_ERR_UNSUPPORTED;
     const int n_split = tmW1 ? 1 : splits;   // the SwiGLU pair needs whole sums before its nonlinearity
     const int total = (a.N + SK_ROWS - 1) / SK_ROWS * n_split;
     const int grid = total < n_sms ? total : n_sms;
-    if (tmW1)
-        gemm_skinny_kernel<true><<<grid, SK_THREADS, SkCfg<true>::SMEM_BYTES, s>>>(tmX, tmW0, *tmW1, a, n_split,
-                                                                                   d_status);
-    else
-        gemm_skinny_kernel<false><<<grid, SK_THREADS, SkCfg<false>::SMEM_BYTES, s>>>(tmX, tmW0, tmW0, a, n_split,
-                                                                                     d_status);
+    // x_rows = rows of tmX's box: 64 (R <= 64) or 128
+    if (x_rows == 64 && a.R <= 64) {
+        if (tmW1)
+            launch_kernel(gemm_skinny_kernel<true, 64>, dim3(grid), dim3(SK_THREADS), SkCfg<true, 64>::SMEM_BYTES, s, pdl,
+                          tmX, tmW0, *tmW1, a, n_split, d_status);
+        else
+            launch_kernel(gemm_skinny_kernel<false, 64>, dim3(grid), dim3(SK_THREADS), SkCfg<false, 64>::SMEM_BYTES, s,
+                          pdl, tmX, tmW0, tmW0, a, n_split, d_status);
+    } else if (x_rows == 128) {
+        if (tmW1)
+            launch_kernel(gemm_skinny_kernel<true, 128>, dim3(grid), dim3(SK_THREADS), SkCfg<true, 128>::SMEM_BYTES, s,
+                          pdl, tmX, tmW0, *tmW1, a, n_split, d_status);
+        else
+            launch_kernel(gemm_skinny_kernel<false, 128>, dim3(grid), dim3(SK_THREADS), SkCfg<false, 128>::SMEM_BYTES, s,
+                          pdl, tmX, tmW0, tmW0, a, n_split, d_status);
+    } else {
+        return KVR_ERR_UNSUPPORTED;
+    }
     return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
 }
 

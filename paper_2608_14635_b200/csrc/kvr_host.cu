@@ -70,6 +70,7 @@ struct kvr_ctx {
     void *tp_user = nullptr;
     // options
     int gemm_impl = 2, attn_impl = 2, profile = 0, probe_mute = 0;
+    int resume_pdl = 1;
     int resume_gemm = 1;           // kv_resume_logits: 1 = weight-streaming GEMM for up to 128 requests, 0 = the rebuild's GEMM
     uint32_t *d_probe = nullptr;   // [2 * PROBE_MAX_BLOCKS]: flags, results
     uint32_t probe_epoch = 0;      // word the current probe publishes; never 0, never reused by the next call
@@ -87,6 +88,8 @@ struct kvr_ctx {
     std::vector<int32_t> last_lens, last_tables;
     int32_t last_width = 0;
     CUtensorMap tm_la_d{}, tm_la_q{}, tm_lm{}, tm_lq{}, tm_lh{};
+    CUtensorMap tm_x_d{}, tm_x_q{}, tm_x_m{};   // l_a and l_m again, box of x_rows rows (weight-streaming GEMM)
+    int x_rows = 128;
 };
 
 namespace {
@@ -588,6 +591,10 @@ int kv_workspace_bind(kvr_ctx *c, void *ws, size_t bytes, int64_t max_chunk_toke
         if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_la_q, c->ws + L.l_a, max_requests, md.q_dim, 128, 64);
         if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_lm, c->ws + L.l_m, max_requests, md.F, 128, 64);
         if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_lq, c->ws + L.l_q, max_requests, md.q_dim, 128, 64);
+        c->x_rows = max_requests <= 64 ? 64 : 128;
+        if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_x_d, c->ws + L.l_a, max_requests, md.d, c->x_rows, 64);
+        if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_x_q, c->ws + L.l_a, max_requests, md.q_dim, c->x_rows, 64);
+        if (st == KVR_OK) st = tc_make_tmap_2d(&c->tm_x_m, c->ws + L.l_m, max_requests, md.F, c->x_rows, 64);
         if (st == KVR_OK) st = tc_make_tmap_f32(&c->tm_lh, c->ws + L.l_h2, max_requests, md.d);
         if (st != KVR_OK) return st;
     }
@@ -626,6 +633,7 @@ int kv_set_option(kvr_ctx *c, const char *name, int64_t value) {
         return write_status_block(c);
     }
     if (!std::strcmp(name, "profile")) { c->profile = (int)value; return KVR_OK; }
+    if (!std::strcmp(name, "resume_overlap")) { c->resume_pdl = (int)value; return KVR_OK; }
     if (!std::strcmp(name, "probe_mute")) { c->probe_mute = (int)value; return KVR_OK; }
     if (!std::strcmp(name, "keep_last_hidden")) { c->keep_last = (int)value; return KVR_OK; }
     return KVR_ERR_INVALID_ARG;
@@ -1049,6 +1057,8 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     // few rows: every projection is bound by reading its weights once, which the weight-streaming GEMM does
     // on all SMs; its K splits leave fp32 partial products that the next kernel sums
     const bool use_sk = use_tc && c->resume_gemm == 1 && R <= GEMM_SKINNY_MAX_ROWS;
+    // on that path every kernel after the first norm may be scheduled while the one before it drains
+    const bool pdl = use_sk && c->resume_pdl;
     if (!use_sk) CU_OK(cudaMemcpyAsync(h, h0, (size_t)R * md.d * sizeof(float), cudaMemcpyDeviceToDevice, s));
     launch_rmsnorm(fp32, h0, c->w[W_LN1][l], a, R, md.d, md.eps, s);
     // q of the final tokens (RoPE at position len - 1); their K/V are already in the arena
@@ -1061,9 +1071,9 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         SkinnyArgs ga{};
         ga.R = R; ga.N = md.q_dim; ga.K = md.d; ga.out_f32 = sk; ga.split_stride = (int64_t)R * md.q_dim;
         ga.ldo = md.q_dim;
-        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WQ][l], nullptr, ga, sp, c->d_status, c->n_sms, s);
+        st = launch_gemm_skinny(c->tm_x_d, c->tm_w[W_WQ][l], nullptr, ga, c->x_rows, sp, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
-        launch_rope_scatter(false, sk, md.q_dim, cs, cm, q_only, c->av, l, true, q, ex, s, sp, ga.split_stride);
+        launch_rope_scatter(false, sk, md.q_dim, cs, cm, q_only, c->av, l, true, q, ex, s, sp, ga.split_stride, pdl);
     } else if (use_tc_q) {
         TcGemmEpilogue ep{};
         set_tc_extras(ep, ex, true);
@@ -1086,7 +1096,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         int max_len = 0;
         for (int r = 0; r < R; ++r) max_len = std::max(max_len, c->last_lens[r]);
         st = launch_attn_decode((const __nv_bfloat16 *)q, d_pos, R, max_len, d_tables, width, md, c->av, l,
-                                (float *)(ws + L.l_part), (__nv_bfloat16 *)a, s);
+                                (float *)(ws + L.l_part), (__nv_bfloat16 *)a, s, pdl);
         if (st != KVR_OK) return st;
     } else if (use_fa) {
         st = launch_attn_fa(c->tm_lq, c->tm_kv, d_tiles, R, d_tables, width, md, c->av, l, (__nv_bfloat16 *)a,
@@ -1105,25 +1115,25 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         int sp = gemm_skinny_splits(md.d, md.q_dim, c->n_sms);
         SkinnyArgs go{};
         go.R = R; go.N = md.d; go.K = md.q_dim; go.out_f32 = sk; go.split_stride = hs; go.ldo = md.d;
-        st = launch_gemm_skinny(c->tm_la_q, c->tm_w[W_WO][l], nullptr, go, sp, c->d_status, c->n_sms, s);
+        st = launch_gemm_skinny(c->tm_x_q, c->tm_w[W_WO][l], nullptr, go, c->x_rows, sp, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
-        launch_add_rmsnorm(false, h0, h, sk, sp, hs, c->w[W_LN2][l], a, R, md.d, md.eps, s);
+        launch_add_rmsnorm(false, h0, h, sk, sp, hs, c->w[W_LN2][l], a, R, md.d, md.eps, s, pdl);
         SkinnyArgs gg{};
         gg.R = R; gg.N = md.F; gg.K = md.d; gg.out_bf16 = (__nv_bfloat16 *)m; gg.ld_bf16 = md.F;
-        st = launch_gemm_skinny(c->tm_la_d, c->tm_w[W_WG][l], &c->tm_w[W_WU][l], gg, 1, c->d_status, c->n_sms, s);
+        st = launch_gemm_skinny(c->tm_x_d, c->tm_w[W_WG][l], &c->tm_w[W_WU][l], gg, c->x_rows, 1, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
         sp = gemm_skinny_splits(md.d, md.F, c->n_sms);
         SkinnyArgs gd{};
         gd.R = R; gd.N = md.d; gd.K = md.F; gd.out_f32 = sk; gd.split_stride = hs; gd.ldo = md.d;
-        st = launch_gemm_skinny(c->tm_lm, c->tm_w[W_WD][l], nullptr, gd, sp, c->d_status, c->n_sms, s);
+        st = launch_gemm_skinny(c->tm_x_m, c->tm_w[W_WD][l], nullptr, gd, c->x_rows, sp, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
-        launch_add_rmsnorm(false, h, h, sk, sp, hs, final_gain, a, R, md.d, md.eps, s);
+        launch_add_rmsnorm(false, h, h, sk, sp, hs, final_gain, a, R, md.d, md.eps, s, pdl);
         CUtensorMap tlm;
         st = tc_make_tmap_2d(&tlm, lm_head, md.V, md.d, 128, 64);
         if (st != KVR_OK) return st;
         SkinnyArgs gl{};
         gl.R = R; gl.N = md.V; gl.K = md.d; gl.out_f32 = logits_out; gl.split_stride = 0; gl.ldo = md.V;
-        st = launch_gemm_skinny(c->tm_la_d, tlm, nullptr, gl, 1, c->d_status, c->n_sms, s);
+        st = launch_gemm_skinny(c->tm_x_d, tlm, nullptr, gl, c->x_rows, 1, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
         return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
     }

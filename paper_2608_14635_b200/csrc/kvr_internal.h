@@ -49,6 +49,33 @@ struct RopeFreq {
     double inv_freq[64];  // base^(-2i/hd), i < hd/2 <= 64
 };
 
+#ifdef __CUDACC__
+// Programmatic dependent launch: a kernel launched with `pdl` may be scheduled while the kernel before it on
+// the stream is still draining; it must not touch global memory before grid_dependency_wait(), which returns
+// once that kernel has completed and its writes are visible (at once when the launch was an ordinary one).
+// Every thread of every block calls it, so a kernel's completion implies the completion of all before it.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel's blocks be scheduled as soon as all of this kernel's blocks have said so or exited.
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                                 Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- plain-FMA kernels (kvr_simt.cu); T selected by `fp32` ----
 void launch_embed_rmsnorm(bool fp32, const void *embed, const void *gain, const ChunkMeta &cm, float *h,
                           void *a, int d, float eps, cudaStream_t s);
@@ -58,7 +85,8 @@ void launch_rmsnorm(bool fp32, const float *h, const void *gain, void *a, int n,
 // h_out may be h_in), then a = rmsnorm(h_out) * gain: the residual add of a row-parallel projection's partial
 // sums folded into the norm that follows it
 void launch_add_rmsnorm(bool fp32, const float *h_in, float *h_out, const float *part, int n_part,
-                        int64_t part_stride, const void *gain, void *a, int n, int d, float eps, cudaStream_t s);
+                        int64_t part_stride, const void *gain, void *a, int n, int d, float eps, cudaStream_t s,
+                        bool pdl = false);
 void launch_rope_table(const int32_t *pos, int n, int hd, const RopeFreq &f, float2 *cs, cudaStream_t s);
 // mode 0: C fp32 [M, ldc] = A W0^T; 1: C fp32 += A W0^T; 2: C (T) = silu(A W0^T) * (A W1^T)
 void launch_gemm_simt(bool fp32, int mode, const void *A, int lda, const void *W0, const void *W1, int ldw,
@@ -75,7 +103,8 @@ struct QkvExtras {
 // elements apart); writes rotated Q (T) and the arena rows.
 void launch_rope_scatter(bool fp32, const float *qkv, int ld, const float2 *cs, const ChunkMeta &cm,
                          const ModelDims &md, const ArenaView &av, int layer, bool want_q, void *q_out,
-                         const QkvExtras &ex, cudaStream_t s, int n_part = 1, int64_t part_stride = 0);
+                         const QkvExtras &ex, cudaStream_t s, int n_part = 1, int64_t part_stride = 0,
+                         bool pdl = false);
 void launch_attn_simt(bool fp32, const void *q, const ChunkMeta &cm, const int32_t *tables, int max_blk,
                       const ModelDims &md, const ArenaView &av, int layer, void *o, cudaStream_t s);
 void launch_gather_rows(const float *h, int d, const int2 *pairs, int n_pairs, float *h_last, cudaStream_t s);
@@ -129,9 +158,11 @@ struct SkinnyArgs {
 };
 int gemm_skinny_init(int device);
 int gemm_skinny_splits(int N, int K, int n_sms);
-// tmX: activation map (box 128 rows x 64), tmW0 / tmW1: weight maps (box 128 x 64); tmW1 non-null = SwiGLU pair
+// tmX: activation map (box x_rows x 64, x_rows = 64 or 128), tmW0 / tmW1: weight maps (box 128 x 64);
+// tmW1 non-null = SwiGLU pair
 int launch_gemm_skinny(const CUtensorMap &tmX, const CUtensorMap &tmW0, const CUtensorMap *tmW1,
-                       const SkinnyArgs &a, int splits, int *d_status, int n_sms, cudaStream_t s);
+                       const SkinnyArgs &a, int x_rows, int splits, int *d_status, int n_sms, cudaStream_t s,
+                       bool pdl = false);
 
 // ---- tensor-core attention (kvr_attn_tc.cu) ----
 int attn_tc_init(int device);
@@ -153,7 +184,7 @@ size_t attn_decode_scratch_bytes(int max_requests, int Hq, int hd);
 // q [R, Hq*hd] bf16, pos[r] = position of the query row (it attends to keys 0..pos[r]); max_len = max(pos) + 1
 int launch_attn_decode(const __nv_bfloat16 *q, const int32_t *pos, int R, int max_len, const int32_t *tables,
                        int max_blk, const ModelDims &md, const ArenaView &av, int layer, float *scratch,
-                       __nv_bfloat16 *o, cudaStream_t s);
+                       __nv_bfloat16 *o, cudaStream_t s, bool pdl = false);
 
 // ---- handover device steps (kvr_handover.cu) ----
 constexpr int PROBE_THREADS = 64, PROBE_ITERS = 1000, PROBE_MAX_BLOCKS = 1024;

@@ -159,6 +159,8 @@ __global__ void __launch_bounds__(256) add_rmsnorm_kernel(const float *__restric
     constexpr int VEC = sizeof(T) == 4 ? 4 : 8;
     extern __shared__ float row[];
     __shared__ float red[32];
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int64_t t = blockIdx.x;
     float ss = 0.f;
     for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
@@ -183,15 +185,16 @@ __global__ void __launch_bounds__(256) add_rmsnorm_kernel(const float *__restric
 }
 
 void launch_add_rmsnorm(bool fp32, const float *h_in, float *h_out, const float *part, int n_part,
-                        int64_t part_stride, const void *gain, void *a, int n, int d, float eps, cudaStream_t s) {
+                        int64_t part_stride, const void *gain, void *a, int n, int d, float eps, cudaStream_t s,
+                        bool pdl) {
     if (n == 0) return;
     const size_t sm = (size_t)d * sizeof(float);
     if (fp32)
-        add_rmsnorm_kernel<float><<<n, 256, sm, s>>>(h_in, h_out, part, n_part, part_stride, (const float *)gain,
-                                                     (float *)a, d, eps);
+        launch_kernel(add_rmsnorm_kernel<float>, dim3(n), dim3(256), sm, s, pdl, h_in, h_out, part, n_part, part_stride,
+                      (const float *)gain, (float *)a, d, eps);
     else
-        add_rmsnorm_kernel<__nv_bfloat16><<<n, 256, sm, s>>>(h_in, h_out, part, n_part, part_stride,
-                                                              (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)a, d, eps);
+        launch_kernel(add_rmsnorm_kernel<__nv_bfloat16>, dim3(n), dim3(256), sm, s, pdl, h_in, h_out, part, n_part,
+                      part_stride, (const __nv_bfloat16 *)gain, (__nv_bfloat16 *)a, d, eps);
 }
 
 void launch_embed_rmsnorm(bool fp32, const void *embed, const void *gain, const ChunkMeta &cm, float *h,
@@ -346,6 +349,8 @@ __global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restri
                                                            const int32_t *__restrict__ slot, int Hq, int Hkv, int hd,
                                                            T *__restrict__ arena_k, int64_t kv_stride,
                                                            bool want_q, T *__restrict__ q_out, QkvExtras ex) {
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int64_t t = blockIdx.x;
     const int half = hd >> 1;
     const float *src0 = qkv + t * ld;
@@ -409,18 +414,18 @@ __global__ void __launch_bounds__(128) rope_scatter_kernel(const float *__restri
 
 void launch_rope_scatter(bool fp32, const float *qkv, int ld, const float2 *cs, const ChunkMeta &cm,
                          const ModelDims &md, const ArenaView &av, int layer, bool want_q, void *q_out,
-                         const QkvExtras &ex, cudaStream_t s, int n_part, int64_t part_stride) {
+                         const QkvExtras &ex, cudaStream_t s, int n_part, int64_t part_stride, bool pdl) {
     if (cm.n == 0) return;
     // one block per row when there are rows enough to fill the GPU, else one block per four heads
     const dim3 grid(cm.n, cm.n >= 1024 ? 1 : (md.Hq + md.Hkv + 3) / 4);
     if (fp32) {
         float *ak = (float *)av.base + (int64_t)layer * av.layer_stride;
-        rope_scatter_kernel<float><<<grid, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak, av.kv_stride,
-                                                         want_q, (float *)q_out, ex);
+        launch_kernel(rope_scatter_kernel<float>, grid, dim3(128), 0, s, pdl, qkv, ld, n_part, part_stride, cs, cm.slot,
+                      md.Hq, md.Hkv, md.hd, ak, av.kv_stride, want_q, (float *)q_out, ex);
     } else {
         __nv_bfloat16 *ak = (__nv_bfloat16 *)av.base + (int64_t)layer * av.layer_stride;
-        rope_scatter_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(qkv, ld, n_part, part_stride, cs, cm.slot, md.Hq, md.Hkv, md.hd, ak,
-                                                                 av.kv_stride, want_q, (__nv_bfloat16 *)q_out, ex);
+        launch_kernel(rope_scatter_kernel<__nv_bfloat16>, grid, dim3(128), 0, s, pdl, qkv, ld, n_part, part_stride, cs,
+                      cm.slot, md.Hq, md.Hkv, md.hd, ak, av.kv_stride, want_q, (__nv_bfloat16 *)q_out, ex);
     }
 }
 

@@ -102,28 +102,29 @@ def test_mid_shape_resume_logits(resume_gemm):
     assert rig.guards_ok()
 
 
-@pytest.mark.parametrize("resume_gemm", [1, 0])
-def test_resume_logits_many_requests_ragged_head_and_repeat(resume_gemm):
-    """37 requests (the request dimension is padded to 48 on the tensor core), a vocabulary that ends
-    inside a 128-row weight tile, and the call made twice after one rebuild: the rows the rebuild
-    kept are only read, so both calls give the same bits."""
+@pytest.mark.parametrize("resume_gemm,n_req", [(1, 37), (0, 37), (1, 66)])
+def test_resume_logits_many_requests_ragged_head_and_repeat(resume_gemm, n_req):
+    """37 or 66 requests (the request dimension is padded to 48 / 80 on the tensor core; above 64 the
+    weight-streaming GEMM stages 128-row activation boxes), a vocabulary that ends inside a 128-row
+    weight tile, and the call made twice after one rebuild: the rows the rebuild kept are only read,
+    so both calls give the same bits."""
     shape = ModelShape("mid-ragged", 2, 1024, 8, 2, 128, 2816, 4100)
     rng = np.random.default_rng(8)
-    lens = tuple(int(x) for x in rng.integers(1, 260, 37))
-    spec = dataclasses.replace(WORKLOADS["cfg2"], n_requests=37, fixed_lens=lens, lognormal_median=None, clip=None,
+    lens = tuple(int(x) for x in rng.integers(1, 260, n_req))
+    spec = dataclasses.replace(WORKLOADS["cfg2"], n_requests=n_req, fixed_lens=lens, lognormal_median=None, clip=None,
                                seed=23)
     wl = make_workload(spec, vocab=shape.vocab)
     batch = wl.rebuild_batch()
-    rig = Rig(shape, "bf16", wl.num_blocks, max_chunk=2048, max_requests=40,
+    rig = Rig(shape, "bf16", wl.num_blocks, max_chunk=2048, max_requests=n_req + 3,
               max_blocks_per_req=batch.tables.shape[1], seed=23)
     assert rig.ctx.kv_set_option("keep_last_hidden", 1) == 0
     assert rig.ctx.kv_set_option("resume_gemm", resume_gemm) == 0
     rig.rebuild(batch)
-    print("37 requests, logits worst rel-L2", _check(rig, batch, 3e-2))
+    print(n_req, "requests, logits worst rel-L2", _check(rig, batch, 3e-2))
     gain, lm = _head(shape, rig.tdtype, rig.dev)
     outs = []
     for _ in range(2):
-        out = torch.full((37, shape.vocab), float("nan"), device=rig.dev)
+        out = torch.full((n_req, shape.vocab), float("nan"), device=rig.dev)
         assert rig.ctx.kv_resume_logits(gain, lm, out) == 0
         assert rig.ctx.kv_sync_status() == 0
         outs.append(out.cpu())
