@@ -5,7 +5,8 @@
 // request are cut into splits, one CTA per (split, kv head, request) reads its K/V rows once for all
 // query heads of the group (GQA), keeps a running softmax per head, and writes an unnormalised
 // partial (max, sum, weighted values); a second small kernel merges the splits of every head.
-// Both products run on warp-level MMAs with the query heads of the group as the rows of the tile.
+// Both products run on warp-level MMAs in transposed form (keys, then head dims, as the rows of the tiles;
+// the query heads of the group as the columns).
 #include "kvr_internal.h"
 
 namespace kvr {
@@ -40,25 +41,32 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&h);
 }
 
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
 // partial layout per (request, q head, split): [HD] weighted values, then max (log2 units) and sum
 //
-// Warp-level MMAs with the GQA group as the M dimension (rows 0..G-1 of a 16-row tile, G <= 8; rows
-// 8..15 stay zero): per 32-key block of a warp
-//   S = Q K^T   four 8-key column tiles x HD/16 k-steps.  The contraction runs over head dims, whose order
-//               is free as long as Q and K agree: lane c = lane % 4 takes dims 32 kp + 8 c .. + 7 of its
-//               key as ONE 16-byte load and feeds them to k-steps 2 kp and 2 kp + 1.
-//   softmax     the accumulator fragment holds, for head lane / 4, the scores of keys 2 c, 2 c + 1 of each
-//               column tile; row statistics are reduced over the four lanes of a row.
-//   O += P V    P's accumulator fragments are already A fragments (two column tiles = one 16-key k-step); V
-//               rows go through shared memory (16-byte cp.async, XOR-swizzled) and ldmatrix.trans.
+// Warp-level MMAs in the transposed form, so that no accumulator row is padding: per 32-key block of a warp
+//   S^T = K Q^T   keys are the M dimension (two 16-key row tiles), the GQA group's heads the N dimension
+//                 (G <= 8 columns; columns >= G see a zero Q).  The contraction runs over head dims, whose
+//                 order is free as long as K and Q agree: lane c = lane % 4 takes dims 32 kp + 8 c .. + 7 of
+//                 its two keys as ONE 16-byte load each and feeds them to k-steps 2 kp and 2 kp + 1.
+//   softmax       a lane holds, for heads 2 c and 2 c + 1, the scores of keys g and g + 8 of each row tile;
+//                 the column statistics are reduced over the eight lanes that share c.
+//   O^T += V^T P^T   head dims are the M dimension (HD / 16 row tiles), heads the N dimension; P's accumulator
+//                 fragments become B fragments by an 8 x 8 transpose across the warp (movmatrix); V rows go
+//                 through shared memory (16-byte cp.async, XOR-swizzled) and ldmatrix.trans as A fragments.
 template <int HD>
-__global__ void __launch_bounds__(DEC_THREADS)
+__global__ void __launch_bounds__(DEC_THREADS, 4)
 attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *__restrict__ pos,
                            const int32_t *__restrict__ tables, int max_blk, int Hq, int Hkv,
                            const __nv_bfloat16 *__restrict__ arena_k, int64_t kv_stride, int block_size,
                            int split_len, int max_splits, float *__restrict__ partial) {
-    constexpr int KP = HD / 32;            // pairs of k-steps of Q K^T
-    constexpr int NT = HD / 8;             // 8-dim column tiles of O
+    constexpr int KP = HD / 32;            // 16-byte pieces of a key row per lane = pairs of k-steps of K Q^T
+    constexpr int DT = HD / 16;            // 16-dim row tiles of O^T
     constexpr int ROW_CHUNKS = HD / 8;     // 16-byte chunks per V row
     grid_dependency_wait();
     grid_launch_dependents();
@@ -75,8 +83,8 @@ attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *_
     // a warp's unnormalised output [G][HD] fp32 goes over its own V buffer once its key blocks are done
     static_assert(DEC_GMAX * HD * 4 <= 32 * HD * 2, "the V buffer holds a warp's partial output");
     const float scale_log2 = rsqrtf((float)HD) * 1.4426950408889634f;
-    // Q fragments of head g (zero rows for g >= G): k-step 2 kp + ks uses dims 32 kp + 8 c + 4 ks + {0,1 | 2,3}
-    uint32_t qa[2 * KP][2];
+    // Q^T fragments of head g (zero for g >= G): k-step 2 kp + ks uses dims 32 kp + 8 c + 4 ks + {0,1 | 2,3}
+    uint32_t qb[2 * KP][2];
     {
         const uint2 *qrow = reinterpret_cast<const uint2 *>(q + (int64_t)r * q_dim + (hk * G + min(g, G - 1)) * HD);
 #pragma unroll
@@ -84,17 +92,19 @@ attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *_
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
                 const uint2 u = qrow[(32 * kp + 8 * c + 4 * ks) / 4];
-                qa[2 * kp + ks][0] = g < G ? u.x : 0u;
-                qa[2 * kp + ks][1] = g < G ? u.y : 0u;
+                qb[2 * kp + ks][0] = g < G ? u.x : 0u;
+                qb[2 * kp + ks][1] = g < G ? u.y : 0u;
             }
     }
     const int32_t *tab = tables + (int64_t)r * max_blk;
     const __nv_bfloat16 *arena_v = arena_k + kv_stride;
     const uint32_t vb = (uint32_t)__cvta_generic_to_shared(&vbuf[warp][0]);
-    float m_run = -INFINITY, l_run = 0.f;   // of head g, over this lane's keys (the sum is reduced over the row's lanes at the end)
-    float o[NT][4];
+    // running statistics of heads 2 c and 2 c + 1: the max is common to the eight lanes that share c, the sum
+    // covers this lane's keys only (reduced over those lanes at the end)
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float o[DT][4];   // O^T: [0], [1] = dim 16 t + g of heads 2 c, 2 c + 1; [2], [3] = dim 16 t + g + 8
 #pragma unroll
-    for (int t = 0; t < NT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+    for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
     for (int kb = k0 + warp * 32; kb < k1; kb += DEC_WARPS * 32) {
         // slot of key kb + lane (keys past the end borrow the last live key: finite rows, probability 0)
         const int key_l = min(kb + lane, k1 - 1);
@@ -109,77 +119,97 @@ attn_decode_partial_kernel(const __nv_bfloat16 *__restrict__ q, const int32_t *_
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
-        // ---- S = Q K^T: four column tiles of 8 keys ----
-        float sacc[4][4];
+        // ---- S^T = K Q^T: two row tiles of 16 keys (rows g and g + 8 of each) ----
+        float st[2][4];
+        uint4 ka[2][KP], kc[2][KP];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            sacc[t][0] = sacc[t][1] = sacc[t][2] = sacc[t][3] = 0.f;
-            const int64_t sl = __shfl_sync(0xffffffffu, slot_l, 8 * t + g);
-            const uint4 *kr = reinterpret_cast<const uint4 *>(arena_k + sl * kv_dim + hk * HD);
-            uint4 kf[KP];
+        for (int mt = 0; mt < 2; ++mt) {
+            const int64_t sa = __shfl_sync(0xffffffffu, slot_l, 16 * mt + g);
+            const int64_t sc8 = __shfl_sync(0xffffffffu, slot_l, 16 * mt + g + 8);
+            const uint4 *ra = reinterpret_cast<const uint4 *>(arena_k + sa * kv_dim + hk * HD);
+            const uint4 *rc = reinterpret_cast<const uint4 *>(arena_k + sc8 * kv_dim + hk * HD);
 #pragma unroll
-            for (int kp = 0; kp < KP; ++kp) kf[kp] = kr[4 * kp + c];
+            for (int kp = 0; kp < KP; ++kp) { ka[mt][kp] = ra[4 * kp + c]; kc[mt][kp] = rc[4 * kp + c]; }
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            st[mt][0] = st[mt][1] = st[mt][2] = st[mt][3] = 0.f;
 #pragma unroll
             for (int kp = 0; kp < KP; ++kp) {
-                mma_bf16_16816(sacc[t], qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, kf[kp].x, kf[kp].y);
-                mma_bf16_16816(sacc[t], qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, kf[kp].z, kf[kp].w);
+                mma_bf16_16816(st[mt], ka[mt][kp].x, kc[mt][kp].x, ka[mt][kp].y, kc[mt][kp].y, qb[2 * kp][0],
+                               qb[2 * kp][1]);
+                mma_bf16_16816(st[mt], ka[mt][kp].z, kc[mt][kp].z, ka[mt][kp].w, kc[mt][kp].w, qb[2 * kp + 1][0],
+                               qb[2 * kp + 1][1]);
             }
         }
-        // ---- softmax statistics of head g over the block's keys ----
-        float sc[4][2], mx = -INFINITY;
+        // ---- softmax statistics of heads 2 c, 2 c + 1 over the block's keys ----
+        float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-        for (int t = 0; t < 4; ++t)
+        for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int key = kb + 8 * t + 2 * c + e;
-                sc[t][e] = key < k1 ? sacc[t][e] * scale_log2 : -INFINITY;
-                mx = fmaxf(mx, sc[t][e]);
+            for (int i = 0; i < 4; ++i) {
+                const int key = kb + 16 * mt + g + 8 * (i >> 1);
+                st[mt][i] = key < k1 ? st[mt][i] * scale_log2 : -INFINITY;
+                mx[i & 1] = fmaxf(mx[i & 1], st[mt][i]);
             }
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m_run, mx);          // finite: the block has at least one live key
-        const float corr = ex2f(m_run - m_new);
-        m_run = m_new;
-        float ps = 0.f;
-        uint32_t pa[4];                                // P as A fragments: tile t -> keys 8 t + 2 c, + 1
+        float corr[2];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            const float p0 = ex2f(sc[t][0] - m_new), p1 = ex2f(sc[t][1] - m_new);
-            ps += p0 + p1;
-            pa[t] = pack2_bf16(p0, p1);
+        for (int e = 0; e < 2; ++e) {
+            mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 4));
+            mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 8));
+            mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 16));
+            const float m_new = fmaxf(m_run[e], mx[e]);   // finite: the block has at least one live key
+            corr[e] = ex2f(m_run[e] - m_new);
+            m_run[e] = m_new;
         }
-        l_run = l_run * corr + ps;
+        uint32_t pb[2][2];   // P^T as B fragments of k-step mt: keys 16 mt + 2 c, + 1 | + 8, + 9 of head g
 #pragma unroll
-        for (int t = 0; t < NT; ++t) { o[t][0] *= corr; o[t][1] *= corr; }
-        // ---- O += P V: two 16-key k-steps x NT column tiles; V fragments by ldmatrix.trans ----
+        for (int mt = 0; mt < 2; ++mt) {
+            const float p0 = ex2f(st[mt][0] - m_run[0]), p1 = ex2f(st[mt][1] - m_run[1]);
+            const float p2 = ex2f(st[mt][2] - m_run[0]), p3 = ex2f(st[mt][3] - m_run[1]);
+            l_run[0] = (mt == 0 ? l_run[0] * corr[0] : l_run[0]) + p0 + p2;
+            l_run[1] = (mt == 0 ? l_run[1] * corr[1] : l_run[1]) + p1 + p3;
+            pb[mt][0] = movmatrix_trans(pack2_bf16(p0, p1));
+            pb[mt][1] = movmatrix_trans(pack2_bf16(p2, p3));
+        }
+#pragma unroll
+        for (int t = 0; t < DT; ++t) { o[t][0] *= corr[0]; o[t][1] *= corr[1]; o[t][2] *= corr[0]; o[t][3] *= corr[1]; }
+        // ---- O^T += V^T P^T: two 16-key k-steps x DT row tiles; V^T fragments by ldmatrix.trans ----
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
-            for (int nt = 0; nt < NT; nt += 2) {
-                // matrix j = lane / 8: keys 16 u + 8 (j & 1) + lane % 8, column tile nt + (j >> 1)
-                const int j = lane >> 3, key = 16 * u + 8 * (j & 1) + (lane & 7), ch = nt + (j >> 1);
+            for (int t = 0; t < DT; ++t) {
+                // matrix j = lane / 8: keys 16 mt + 8 (j >> 1) + lane % 8, dims 16 t + 8 (j & 1) .. + 7
+                const int j = lane >> 3, key = 16 * mt + 8 * (j >> 1) + (lane & 7), ch = 2 * t + (j & 1);
                 const uint32_t addr = vb + (uint32_t)(key * ROW_CHUNKS + (ch ^ (key & 7))) * 16u;
-                uint32_t b0, b1, b2, b3;
+                uint32_t a0, a1, a2, a3;
                 asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                             : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3) : "r"(addr));
-                mma_bf16_16816(o[nt], pa[2 * u], 0u, pa[2 * u + 1], 0u, b0, b1);
-                mma_bf16_16816(o[nt + 1], pa[2 * u], 0u, pa[2 * u + 1], 0u, b2, b3);
+                             : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+                mma_bf16_16816(o[t], a0, a1, a2, a3, pb[mt][0], pb[mt][1]);
             }
         }
         __syncwarp();   // the V buffer is refilled at the top of the next block
     }
     // ---- merge the four warps (a warp that saw no key block has m = -inf, l = 0) ----
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (g < G) {
-        float *ro = reinterpret_cast<float *>(&vbuf[warp][0]) + g * HD;
-        if (c == 0) { red_m[warp][g] = m_run; red_l[warp][g] = l_run; }
 #pragma unroll
-        for (int t = 0; t < NT; ++t) {
-            ro[8 * t + 2 * c] = o[t][0];
-            ro[8 * t + 2 * c + 1] = o[t][1];
+    for (int e = 0; e < 2; ++e) {
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+    }
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int hh = 2 * c + e;
+        if (hh < G) {
+            float *ro = reinterpret_cast<float *>(&vbuf[warp][0]) + hh * HD;
+            if (g == 0) { red_m[warp][hh] = m_run[e]; red_l[warp][hh] = l_run[e]; }
+#pragma unroll
+            for (int t = 0; t < DT; ++t) {
+                ro[16 * t + g] = o[t][e];
+                ro[16 * t + g + 8] = o[t][2 + e];
+            }
         }
     }
     __syncthreads();
