@@ -130,3 +130,29 @@ def test_resume_logits_many_requests_ragged_head_and_repeat(resume_gemm, n_req):
         outs.append(out.cpu())
     assert torch.equal(outs[0], outs[1])
     assert rig.guards_ok()
+
+
+def test_resume_logits_more_requests_than_the_streaming_gemm_takes():
+    """Above 128 requests the projections go through the rebuild's GEMM; the logits still match the oracle
+    and the call can still be repeated."""
+    rng = np.random.default_rng(9)
+    n_req = 131
+    lens = tuple(int(x) for x in rng.integers(1, 40, n_req))
+    spec = dataclasses.replace(WORKLOADS["cfg1"], n_requests=n_req, fixed_lens=lens, lognormal_median=None, clip=None,
+                               num_blocks=600, seed=29)
+    wl = make_workload(spec, vocab=TINY.vocab)
+    batch = wl.rebuild_batch()
+    rig = Rig(TINY, "bf16", wl.num_blocks, max_chunk=1024, max_requests=n_req, max_blocks_per_req=batch.tables.shape[1],
+              seed=29)
+    assert rig.ctx.kv_set_option("keep_last_hidden", 1) == 0
+    rig.rebuild(batch)
+    print(n_req, "requests, logits worst rel-L2", _check(rig, batch, 2e-2))
+    gain, lm = _head(TINY, rig.tdtype, rig.dev)
+    outs = []
+    for _ in range(2):
+        out = torch.full((n_req, TINY.vocab), float("nan"), device=rig.dev)
+        assert rig.ctx.kv_resume_logits(gain, lm, out) == 0
+        assert rig.ctx.kv_sync_status() == 0
+        outs.append(out.cpu())
+    assert torch.equal(outs[0], outs[1])
+    assert rig.guards_ok()
