@@ -349,7 +349,7 @@ def compare_readback(rig: Rig, batch, kv_by_request: Dict[int, Tuple[np.ndarray,
     return worst
 
 
-def judge_rows(label: str, layer: int, name: str, got: np.ndarray, want: np.ndarray, floor: Optional[np.ndarray],
+def assess_rows(label: str, layer: int, name: str, got: np.ndarray, want: np.ndarray, floor: Optional[np.ndarray],
                rel_tol: float, abs_tol: float, table: list, failures: list) -> None:
     """The same per-layer bound as compare_readback for one set of rows: the stated tolerance, or --
     where the oracle's bf16-storage pass (`floor`) is itself beyond it -- at most the margins above

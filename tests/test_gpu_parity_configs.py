@@ -18,7 +18,7 @@ import torch
 import oracle
 from synth import (MODEL_SHAPES, WORKLOADS, BENCH_CHUNK_TOKENS, make_workload, make_weights, fill_sentinel,
                    split_waves)
-from kvr_harness import (Rig, compare_readback, check_untouched_on_device, block_checksums, report_table, track, judge_rows,
+from kvr_harness import (Rig, compare_readback, check_untouched_on_device, block_checksums, report_table, track, assess_rows,
                          oracle_weights, oracle_definition_and_floor)
 
 pytestmark = pytest.mark.gpu
@@ -65,8 +65,8 @@ def _long_range_check(rig, table, tokens, chunk, seed, label):
     for layer, (wk, wv), (fk, fv), sel in ((0, (K0, V0), (K0f, V0f), slice(None)), (1, (K1, V1), (K1f, V1f), rows)):
         gk, gv = _fetch_rows(rig, layer, table, n)
         assert not np.isnan(gk).any() and not np.isnan(gv).any()
-        judge_rows(label, layer, "K", gk[sel], wk, fk, BF16_REL, BF16_ABS, table_out, failures)
-        judge_rows(label, layer, "V", gv[sel], wv, fv, BF16_REL, BF16_ABS, table_out, failures)
+        assess_rows(label, layer, "K", gk[sel], wk, fk, BF16_REL, BF16_ABS, table_out, failures)
+        assess_rows(label, layer, "V", gv[sel], wv, fv, BF16_REL, BF16_ABS, table_out, failures)
     report_table(label, table_out)
     assert not failures, "; ".join(failures)
     return rows
