@@ -59,7 +59,15 @@ def test_tiny_resume_logits(dtype, gemm, attn, tol):
     worst = _check(rig, batch, tol)
     # keeping the hidden rows changes nothing in the arena
     kv = oracle_kv(weights_to_cpu(rig.weights), TINY, batch)
+    gain, lm = _head(TINY, rig.tdtype, rig.dev)
+    first = torch.zeros(len(batch.lens), TINY.vocab, device=rig.dev)
+    assert rig.ctx.kv_resume_logits(gain, lm, first) == 0
     compare_rebuilt(rig, batch, kv, 1e-4 if dtype == "fp32" else 1e-2, 1e-3 if dtype == "fp32" else 6e-2)
+    # the read-backs above put their own tables into the workspace: the next call brings the rebuild's back
+    again = torch.zeros_like(first)
+    assert rig.ctx.kv_resume_logits(gain, lm, again) == 0
+    assert rig.ctx.kv_sync_status() == 0
+    assert torch.equal(first, again)
     assert rig.guards_ok()
     print(f"tiny {dtype} gemm={gemm} attn={attn} logits worst rel-L2", worst)
 
