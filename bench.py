@@ -426,7 +426,7 @@ def main():
                     help="tokens per workspace chunk (default: synth.BENCH_CHUNK_TOKENS = 18944)")
     ap.add_argument("--profile-steps", type=int, default=2,
                     help="steps of the separate per-kernel timing pass (at most --steps)")
-    ap.add_argument("--cpu-tokens", type=int, default=256)
+    ap.add_argument("--cpu-tokens", type=int, default=384)
     ap.add_argument("--ref-tokens", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--variant", default="none", choices=["none", "bias", "qknorm"],
