@@ -166,7 +166,7 @@ def test_cfg5_32b_shape_two_waves():
     is left of the device and the requests go in waves that reuse the same block ids.  Per wave, on
     the device: all 64 layers rebuilt through the benchmark's chunk size, untouched rows bit-exact
     against the fill (the arena is refilled between waves, so a row of wave 1 cannot pass for a row of
-    wave 2), a second rebuild reproduces every block checksum.  Oracle: wave 1, a 128-token truncation
+    wave 2), and for the first wave a second rebuild reproduces every block checksum.  Oracle: wave 1, a 128-token truncation
     of one request at full depth (definition and bf16 floor); wave 2, the same to 16 layers only (the
     host cost of 64 layers of this shape is about a minute per pass); and layers 0-1 of the longest
     request on sampled rows across all its chunk boundaries."""
@@ -240,9 +240,10 @@ def test_cfg5_32b_shape_two_waves():
                               "cfg5_long_range_layers01")
             did_long = True
             lap("long-range rows")
-        rig.rebuild(b)                                      # idempotence at full size, bit for bit
-        assert torch.equal(block_checksums(rig), c_first)
-        lap("second rebuild + checksums")
+        if wi == 0:                                         # idempotence at full size, bit for bit (one wave: half a minute each)
+            rig.rebuild(b)
+            assert torch.equal(block_checksums(rig), c_first)
+            lap("second rebuild + checksums")
         del c_first
     assert did_long
     assert rig.guards_ok()
