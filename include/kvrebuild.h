@@ -130,8 +130,10 @@ int kv_variant_bind(kvr_ctx *ctx, const kv_proj_variant *variant);
  *   contains no collective and never touches another rank's memory.
  * tp_world = 1 (or config NULL) clears the sharding.  Call after kv_weights_bind and before
  * kv_workspace_bytes / kv_workspace_bind (the workspace gains one fp32 [chunk, d_model] buffer).
- * All ranks must be given the same batch, chunk size and options.  kv_resume_logits is not
- * available under TP (KVR_ERR_UNSUPPORTED). */
+ * All ranks must be given the same batch, chunk size and options.  kv_resume_logits works under TP
+ * too: every rank finishes the last layer with its slices, calls the callback twice (after the output
+ * and the down projection, on up to 8 * R * d_model values) and multiplies by the whole LM head, so
+ * every rank ends with the same logits. */
 typedef int (*kv_allreduce_fn)(void *buf_dev, int64_t count, void *stream, void *user);
 typedef struct {
     int32_t tp_world, tp_rank;

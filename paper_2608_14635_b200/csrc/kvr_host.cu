@@ -1011,7 +1011,6 @@ int kv_sync_status(kvr_ctx *c, void *stream) {
 int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, float *logits_out, void *stream) {
     if (!c || !final_gain || !lm_head || !logits_out) return KVR_ERR_INVALID_ARG;
     if (!c->arena_bound || !c->weights_bound || !c->ws_bound) return KVR_ERR_NOT_BOUND;
-    if (c->tp_world > 1) return KVR_ERR_UNSUPPORTED;   // the last layer's reductions and a sharded head are not built
     if (!c->have_last) return KVR_ERR_NOT_BOUND;   // no rebuild with "keep_last_hidden" came before
     const ModelDims &md = c->md;
     const bool fp32 = is_fp32(c);
@@ -1058,7 +1057,14 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
     // on all SMs; its K splits leave fp32 partial products that the next kernel sums
     const bool use_sk = use_tc && c->resume_gemm == 1 && R <= GEMM_SKINNY_MAX_ROWS;
     // on that path every kernel after the first norm may be scheduled while the one before it drains
-    const bool pdl = use_sk && c->resume_pdl;
+    // Tensor-parallel ranks: the output and down projections leave this rank's partial sums in `sk`, the callback
+    // sums them over the ranks, the norm that follows adds them to the residual; the head is whole on every rank.
+    const bool tp = c->tp_world > 1;
+    auto tp_sum = [&](int64_t count) -> int {
+        if (!tp) return KVR_OK;
+        return c->tp_allreduce(sk, count, (void *)s, c->tp_user) == 0 ? KVR_OK : KVR_ERR_CUDA;
+    };
+    const bool pdl = use_sk && c->resume_pdl && !tp;   // the callback's work sits between the kernels of the chain
     if (!use_sk) CU_OK(cudaMemcpyAsync(h, h0, (size_t)R * md.d * sizeof(float), cudaMemcpyDeviceToDevice, s));
     launch_rmsnorm(fp32, h0, c->w[W_LN1][l], a, R, md.d, md.eps, s);
     // q of the final tokens (RoPE at position len - 1); their K/V are already in the arena
@@ -1117,6 +1123,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         go.R = R; go.N = md.d; go.K = md.q_dim; go.out_f32 = sk; go.split_stride = hs; go.ldo = md.d;
         st = launch_gemm_skinny(c->tm_x_q, c->tm_w[W_WO][l], nullptr, go, c->x_rows, sp, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
+        if ((st = tp_sum(sp * hs)) != KVR_OK) return st;
         launch_add_rmsnorm(false, h0, h, sk, sp, hs, c->w[W_LN2][l], a, R, md.d, md.eps, s, pdl);
         SkinnyArgs gg{};
         gg.R = R; gg.N = md.F; gg.K = md.d; gg.out_bf16 = (__nv_bfloat16 *)m; gg.ld_bf16 = md.F;
@@ -1127,6 +1134,7 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         gd.R = R; gd.N = md.d; gd.K = md.F; gd.out_f32 = sk; gd.split_stride = hs; gd.ldo = md.d;
         st = launch_gemm_skinny(c->tm_x_m, c->tm_w[W_WD][l], nullptr, gd, c->x_rows, sp, c->d_status, c->n_sms, s, pdl);
         if (st != KVR_OK) return st;
+        if ((st = tp_sum(sp * hs)) != KVR_OK) return st;
         launch_add_rmsnorm(false, h, h, sk, sp, hs, final_gain, a, R, md.d, md.eps, s, pdl);
         CUtensorMap tlm;
         st = tc_make_tmap_2d(&tlm, lm_head, md.V, md.d, 128, 64);
@@ -1137,17 +1145,25 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         if (st != KVR_OK) return st;
         return cudaGetLastError() == cudaSuccess ? KVR_OK : KVR_ERR_CUDA;
     }
+    const int64_t hs = (int64_t)R * md.d;
     if (use_tc) {
         TcGemmEpilogue ep{};
-        ep.mode = TC_RESID; ep.M = R; ep.N = md.d; ep.K = md.q_dim; ep.c_f32 = h; ep.ldc = md.d;
+        ep.mode = tp ? TC_STORE_F32 : TC_RESID; ep.M = R; ep.N = md.d; ep.K = md.q_dim; ep.c_f32 = tp ? sk : h;
+        ep.ldc = md.d;
         ep.n_b = 1; ep.b_rows[0] = md.d;
         CUtensorMap tbm[3] = {c->tm_w[W_WO][l], c->tm_w[W_WO][l], c->tm_w[W_WO][l]};
-        st = launch_gemm_tc(c->tm_la_q, tbm, ep, c->d_status, c->n_sms, s, &c->tm_lh, c->gemm_impl == 2);
+        st = launch_gemm_tc(c->tm_la_q, tbm, ep, c->d_status, c->n_sms, s, tp ? nullptr : &c->tm_lh, c->gemm_impl == 2);
         if (st != KVR_OK) return st;
     } else {
-        launch_gemm_simt(fp32, 1, a, md.q_dim, c->w[W_WO][l], nullptr, md.q_dim, R, md.d, md.q_dim, h, md.d, s);
+        launch_gemm_simt(fp32, tp ? 0 : 1, a, md.q_dim, c->w[W_WO][l], nullptr, md.q_dim, R, md.d, md.q_dim,
+                         tp ? sk : h, md.d, s);
     }
-    launch_rmsnorm(fp32, h, c->w[W_LN2][l], a, R, md.d, md.eps, s);
+    if (tp) {
+        if ((st = tp_sum(hs)) != KVR_OK) return st;
+        launch_add_rmsnorm(fp32, h, h, sk, 1, 0, c->w[W_LN2][l], a, R, md.d, md.eps, s);
+    } else {
+        launch_rmsnorm(fp32, h, c->w[W_LN2][l], a, R, md.d, md.eps, s);
+    }
     if (use_tc) {
         TcGemmEpilogue ep{};
         ep.mode = TC_SWIGLU; ep.M = R; ep.N = 2 * md.F; ep.K = md.d;
@@ -1156,17 +1172,23 @@ int kv_resume_logits(kvr_ctx *c, const void *final_gain, const void *lm_head, fl
         st = launch_gemm_tc(c->tm_la_d, tbm, ep, c->d_status, c->n_sms, s, nullptr, c->gemm_impl == 2);
         if (st != KVR_OK) return st;
         TcGemmEpilogue e2{};
-        e2.mode = TC_RESID; e2.M = R; e2.N = md.d; e2.K = md.F; e2.c_f32 = h; e2.ldc = md.d;
+        e2.mode = tp ? TC_STORE_F32 : TC_RESID; e2.M = R; e2.N = md.d; e2.K = md.F; e2.c_f32 = tp ? sk : h;
+        e2.ldc = md.d;
         e2.n_b = 1; e2.b_rows[0] = md.d;
         CUtensorMap tb2[3] = {c->tm_w[W_WD][l], c->tm_w[W_WD][l], c->tm_w[W_WD][l]};
-        st = launch_gemm_tc(c->tm_lm, tb2, e2, c->d_status, c->n_sms, s, &c->tm_lh, c->gemm_impl == 2);
+        st = launch_gemm_tc(c->tm_lm, tb2, e2, c->d_status, c->n_sms, s, tp ? nullptr : &c->tm_lh, c->gemm_impl == 2);
         if (st != KVR_OK) return st;
     } else {
         launch_gemm_simt(fp32, 2, a, md.d, c->w[W_WG][l], c->w[W_WU][l], md.d, R, md.F, md.d, m, md.F, s);
-        launch_gemm_simt(fp32, 1, m, md.F, c->w[W_WD][l], nullptr, md.F, R, md.d, md.F, h, md.d, s);
+        launch_gemm_simt(fp32, tp ? 0 : 1, m, md.F, c->w[W_WD][l], nullptr, md.F, R, md.d, md.F, tp ? sk : h, md.d, s);
     }
     // final norm and LM head
-    launch_rmsnorm(fp32, h, final_gain, a, R, md.d, md.eps, s);
+    if (tp) {
+        if ((st = tp_sum(hs)) != KVR_OK) return st;
+        launch_add_rmsnorm(fp32, h, h, sk, 1, 0, final_gain, a, R, md.d, md.eps, s);
+    } else {
+        launch_rmsnorm(fp32, h, final_gain, a, R, md.d, md.eps, s);
+    }
     if (use_tc) {
         CUtensorMap tlm;
         st = tc_make_tmap_2d(&tlm, lm_head, md.V, md.d, 128, 64);

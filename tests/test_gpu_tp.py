@@ -95,6 +95,7 @@ def test_tp2_rebuild_matches_unsharded_oracle(dtype, gemm, attn):
         if dtype == "bf16":
             rig.set_impl(gemm, attn)
         assert rig.ctx.kv_tp_bind(2, rank, summer.callback(rank)) == 0
+        assert rig.ctx.kv_set_option("keep_last_hidden", 1) == 0
         assert rig.kb.STATUS[rig.ctx.kv_rebuild(batch.tokens, batch.lens, batch.tables)] == "KVR_ERR_NOT_BOUND"
         rig.bind_workspace(256, 4, tables.shape[1])               # the layout gained the partial-sum buffer
         rigs.append(rig)
@@ -130,8 +131,30 @@ def test_tp2_rebuild_matches_unsharded_oracle(dtype, gemm, attn):
         assert np.array_equal(rig.arena_bits(), first[rank])
         assert rig.guards_ok()
         print(f"tp rank {rank} {dtype}: kv heads {h0}..{h1 - 1}, worst", worst)
-    # resume logits are not offered under TP
-    g = torch.ones(shape.d_model, dtype=tdt, device="cuda:0")
-    lm = torch.zeros(shape.vocab, shape.d_model, dtype=tdt, device="cuda:0")
-    out = torch.zeros(3, shape.vocab, device="cuda:0")
-    assert kb.STATUS[rigs[0].ctx.kv_resume_logits(g, lm, out)] == "KVR_ERR_UNSUPPORTED"
+    # next-token logits under TP: both ranks finish the last layer for the final tokens with their slices, the two
+    # row-parallel products are summed through the same callback, the head is whole on every rank
+    g = torch.Generator().manual_seed(5)
+    gain = (1.0 + 0.02 * torch.randn(shape.d_model, generator=g)).to(tdt).to("cuda:0")
+    lm = (0.02 * torch.randn(shape.vocab, shape.d_model, generator=g)).to(tdt).to("cuda:0")
+    outs = [torch.full((3, shape.vocab), float("nan"), device="cuda:0") for _ in range(2)]
+    calls_before = list(summer.calls)
+
+    def resume(rank):
+        torch.cuda.set_device(0)
+        status[rank] = rigs[rank].ctx.kv_resume_logits(gain, lm, outs[rank], streams[rank])
+
+    ths = [threading.Thread(target=resume, args=(r,)) for r in range(2)]
+    [t.start() for t in ths]
+    [t.join(120) for t in ths]
+    assert status == [0, 0], status
+    for r in range(2):
+        assert rigs[r].ctx.kv_sync_status(streams[r]) == 0
+    assert [summer.calls[r] - calls_before[r] for r in range(2)] == [2, 2]
+    assert torch.equal(outs[0], outs[1])                          # the summed residuals are the same bits on both ranks
+    got = outs[0].double().cpu().numpy()
+    off = np.concatenate([[0], np.cumsum(lens)])
+    for r in range(3):
+        want = oracle.resume_logits(w_cpu, shape, batch.tokens[off[r]:off[r + 1]], gain.cpu(), lm.cpu())
+        err = float(np.linalg.norm(got[r] - want) / np.linalg.norm(want))
+        assert err <= (1e-4 if dtype == "fp32" else 2e-2), (r, err)
+    print(f"tp {dtype}: resume logits match the unsharded oracle")
