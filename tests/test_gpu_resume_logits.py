@@ -111,9 +111,9 @@ def test_mid_shape_resume_logits(resume_gemm):
     assert rig.guards_ok()
 
 
-@pytest.mark.parametrize("resume_gemm,n_req", [(1, 37), (0, 37), (1, 66)])
+@pytest.mark.parametrize("resume_gemm,n_req", [(1, 37), (0, 37), (1, 66), (1, 1), (1, 17)])
 def test_resume_logits_many_requests_ragged_head_and_repeat(resume_gemm, n_req):
-    """37 or 66 requests (the request dimension is padded to 48 / 80 on the tensor core; above 64 the
+    """1, 17, 37 or 66 requests (the request dimension is padded to 16, 32, 48, 80 on the tensor core; above 64 the
     weight-streaming GEMM stages 128-row activation boxes), a vocabulary that ends inside a 128-row
     weight tile, and the call made twice after one rebuild: the rows the rebuild kept are only read,
     so both calls give the same bits."""
