@@ -103,7 +103,7 @@ def test_cfg4_partial_recovery_full_size():
     every block owned only by the seeded 25 % subset scribbled over (after a failure a pool may hold
     partly written entries: paper Sec. 2.3); the subset alone rebuilt; every block no subset request
     references must keep its checksum in every layer; two rebuilt requests -- one inside a
-    shared-prefix group -- compared with the oracle at full depth on 256-token truncations."""
+    shared-prefix group -- compared with the oracle at full depth on 128-token truncations."""
     torch.cuda.empty_cache()
     spec = WORKLOADS["cfg4"]
     shape = MODEL_SHAPES[spec.model]
@@ -147,7 +147,7 @@ def test_cfg4_partial_recovery_full_size():
         st, k, v = rig.ctx.kv_readback(s.n_layers - 1, sub.tables[i], min(int(sub.lens[i]), 4096))
         assert st == 0 and not ((k & 0x7FFF) > 0x7F80).any() and not ((v & 0x7FFF) > 0x7F80).any()
 
-    # oracle, full depth, 256-token truncations: one request of a shared-prefix group, one outside
+    # oracle, full depth, 128-token truncations: one request of a shared-prefix group, one outside
     off = np.concatenate([[0], np.cumsum(sub.lens)])
     in_group = [i for i, r in enumerate(wl.rebuild_ids.tolist()) if wl.group_of[r] >= 0]
     outside = [i for i, r in enumerate(wl.rebuild_ids.tolist()) if wl.group_of[r] < 0]
@@ -155,7 +155,7 @@ def test_cfg4_partial_recovery_full_size():
     w = oracle_weights(rig.weights)
     kv, floor = {}, {}
     for i in (in_group[0], outside[0]):
-        toks = sub.tokens[off[i]:off[i] + 256]
+        toks = sub.tokens[off[i]:off[i] + 128]
         kv[i], floor[i] = oracle_definition_and_floor(w, shape, toks)
     worst = compare_readback(rig, sub, kv, BF16_REL, BF16_ABS, kv_format_floor=floor, label="cfg4_full_depth")
     print("cfg4 full-depth sampled", {k: v for k, v in worst.items() if k != "table"})
